@@ -221,7 +221,7 @@ sc_status sc_matmul_cbsg(sc_ctx *ctx, const float *A, const float *W, int64_t M,
 sc_status sc_cbsg_scc(sc_ctx *ctx, const int32_t *Ta, const int32_t *Tw, int64_t n, int32_t L, uint64_t seed,
                       uint32_t stream_id, int32_t *counts, double *scc, void *ws, size_t ws_bytes, void *stream);
 
-/* ---- Sec. 3.3: Gaussian surrogate of an SC product -------------------------------------------- */
+/* ---- Sec. 3.2: Gaussian surrogate of an SC product -------------------------------------------- */
 /* out_ij = Y_ij (1 + alpha(L_i) Z_ij), Z_ij independent standard normal, alpha(L) = coeff / L: the cheap
  * stand-in the paper uses to sweep model-level tolerance without running the stochastic matmul.
  * SC_SURROGATE_COEFF reproduces the paper's printed table of alpha against L.  Y and out are device
@@ -275,8 +275,20 @@ int32_t sc_selftest_comparator(void);
  * number of mismatches (0 = correct).  Runs on the CPU.                                                            */
 int32_t sc_selftest_expansion(void);
 
-/* Device micro-benchmarks of the units the GEMM cores are bound by.  Every loop and every wait in them is
- * bounded; they allocate nothing and touch only the context's scratch block.
+/* Device check of the failure-detection path: every wait of the tensor-core core on an mbarrier is bounded (a clock
+ * limit and an abort flag shared by the roles of a CTA); a wait that runs out records SC_ERR_TIMEOUT in the device
+ * status word and where it happened beside it, raises the abort flag, and the kernel returns normally.  This call
+ * makes that happen in a kernel of one small CTA that does nothing else: one warp waits, with the core's own wait
+ * routine and a limit of `limit_cycles` SM clocks (1 .. 2e9), on a barrier that is never signalled; a second warp
+ * waits with the default limit and must leave through the abort flag.  Synchronises.  site_host (HOST, 3 ints)
+ * receives the recorded site word (site 99 | warp << 8 | CTA << 16) and its two counters; cycles_host (HOST, 2
+ * int64) the SM clocks each warp waited (-1 if its wait was satisfied, which cannot happen).  The status word
+ * stays set: the next sc_device_status returns SC_ERR_TIMEOUT and clears it.  Nothing else is disturbed.       */
+sc_status sc_selftest_bounded_wait(sc_ctx *ctx, int64_t limit_cycles, int32_t *site_host, int64_t *cycles_host);
+
+/* Device micro-benchmarks of the units the GEMM cores are bound by (the measured denominators of the reported roofline
+ * fractions).  Every loop and every wait in them is bounded; they allocate nothing and touch only the context's
+ * scratch block.
  *
  * kind 0..7 -- register-only instruction-mix loops, `iters` trips per thread on every SM.  0 POPC only,
  *   1 LOP3 only, 2 LOP3+POPC+IADD (the plain core mix), 3 carry-save mix (3 words -> 2 POPC), 4 IADD3 only,
@@ -285,28 +297,11 @@ int32_t sc_selftest_expansion(void);
  *   operations of the named kind executed on the whole GPU (mixes: gate evaluations of 32 stream bit-ops
  *   each; kind 7: multiply-accumulates).
  *
- * kind 8 + v -- issue rate of the 128 x N x 32 tensor-memory MMA with 8-bit operands (the tensor-core core issues the
- *   4-bit block-scaled form of the same instruction, 64 deep, at twice that rate), one CTA per SM, `iters` MMAs in
- *   groups of four.  Bits of v: 0 = A operand from tensor memory instead of shared memory,
- *   1 = 8-bit float operands instead of 8-bit integers, 2-3 = N (0: 256, 1: 192, 2: 128), 4-7 = commit to
- *   an mbarrier after every that many groups (0: once at the end), 8-11 = hundreds of SM clocks of
- *   thread-side delay per group (bit 12: placed before the commit instead of after), 13-17 = extra
- *   per-group operations (1 fence, 2 barrier test, 4 barrier try-wait).  *ms_out = SM CLOCKS / 1e6 of the
- *   slowest SM (not milliseconds), *words_out = multiply-accumulates PER SM.
- *
- * kind 1000000 + 10 * mode + busy -- clocks per iteration (*ms_out, in clocks) of one warp doing the
- *   expander-side operation `mode` (1 four tensor-memory stores + wait + fence, 2 eight 16-byte shared
- *   stores + async-proxy fence, 4 one barrier try-wait; each followed by one mbarrier arrive) while the
- *   tensor pipe is idle (busy 0) or running MMAs back to back (busy 1).
- *
- * kind 2000000 + 100 * mode + n_side -- clocks per MMA (*ms_out) of one issuer running `iters` MMAs while
- *   n_side (0..24) other warps loop on operation `mode` (1 tensor-memory stores, 2 shared stores, 3 shared
- *   stores + async-proxy fence, 4 the fence alone, 5 mbarrier arrive, 6 mbarrier try-wait, 7 tensor-memory
- *   loads, 8 shared loads).
- *
- * kind 4000000 + 1000 * d_col + a_col -- clocks per MMA with the accumulator at tensor-memory column d_col
- *   and the A operand at column a_col (placement sensitivity; d_col + 192 <= 512, a_col + 64 <= 512, no
- *   overlap -- anything else is SC_ERR_ARG).                                                           */
+ * kind 8, 9 -- issue-rate ceiling of the tensor-core core's instruction: one thread per SM issues `iters` (rounded up
+ *   to a multiple of 8, at most 2^22) block-scaled 4-bit MMAs, 128 x N x 64 with N = 192 (kind 8, the core's tile) or 256
+ *   (kind 9), A operand and scale factors in tensor memory, B operand in shared memory, back to back on zero-filled
+ *   operands, and waits (bounded) for the last one.  *ms_out = SM CLOCKS / 1e6 of the slowest SM (not milliseconds),
+ *   *words_out = multiply-accumulates PER SM; their ratio / 1e6 is multiply-accumulates per clock per SM.        */
 sc_status sc_microbench(sc_ctx *ctx, int32_t kind, int32_t iters, float *ms_out, double *words_out);
 
 #ifdef __cplusplus

@@ -30,7 +30,7 @@
  *                          thresholded stream length at a matched average budget.
  *   sco_ladder_lengths     Sec. 4.4 inference rule with an explicit ladder and
  *                          threshold list: first level whose threshold is reached.
- *   sco_surrogate_noise    Sec. 3.3: Gaussian-perturbed stand-in for an SC product,
+ *   sco_surrogate_noise    Sec. 3.2: Gaussian-perturbed stand-in for an SC product,
  *                          Y (1 + alpha(L) Z) with alpha(L) = coeff / L.
  *   sco_cbsg_*             Sec. 4.2 / Appendix A.1: Sobol-8 streams with conditional
  *                          bitstream generation, cycle by cycle (a reading: the paper
@@ -114,6 +114,32 @@ int32_t sco_boundary_unipolar(float v, int32_t *sign)
     if (t < 0) t = 0;
     if (t > 256) t = 256;
     return (int32_t)t;
+}
+
+/* Sec. 4.2 ("Datapath"), the two-step variant: operands first go to the int8 */
+/* grid, x_hat = round(127 v) in -127..127 (Sec. 3.1: q_max = 2^(b-1) - 1 with */
+/* b = 8), and the grid point is then converted to one of the 257 boundaries.  */
+/* The paper does not print the conversion; reading: the boundary nearest to   */
+/* the offset grid point (x_hat + q_max) / (2 q_max) of Sec. 3.1 on the 0..256 */
+/* scale, T = round((x_hat + 127) 128 / 127).  127 is odd, so no grid point    */
+/* falls half-way between two boundaries and the rounding is plain integer     */
+/* arithmetic.  Unipolar: magnitude |x_hat| in 0..127 -> T = round(|x_hat| 256 / 127). */
+int32_t sco_boundary_bipolar_int8(float v)
+{
+    volatile float scaled = v * 127.0f;
+    long q = lrintf(scaled);                  /* round half to even (default mode) */
+    if (q < -127) q = -127;
+    if (q > 127) q = 127;
+    return (int32_t)(((q + 127) * 256 + 127) / 254);
+}
+
+int32_t sco_boundary_unipolar_int8(float v, int32_t *sign)
+{
+    *sign = (v < 0.0f) ? 1 : 0;
+    volatile float scaled = fabsf(v) * 127.0f;
+    long q = lrintf(scaled);
+    if (q > 127) q = 127;
+    return (int32_t)((q * 512 + 127) / 254);
 }
 
 /* ------------------------------------------------------------------------- */
@@ -217,6 +243,14 @@ void sco_row_absmax(const float *X, int64_t rows, int64_t cols, float *g)
 /*   L_sel[nr*nc]-free form : every selected element gets `L` positions.     */
 /*   bits[(a*nc + b)*L + l] : 0/1, T[a*nc+b], sign[a*nc+b] (unipolar only).   */
 /* ------------------------------------------------------------------------- */
+/* quant: 0 = straight onto the 257-boundary grid, 1 = int8 grid first (Sec. 4.2). */
+int32_t sco_encode_quant(const float *X, int64_t rows, int64_t cols,
+                         const int64_t *row_sel, int64_t nr, const int64_t *col_sel, int64_t nc,
+                         int32_t tensor_id, int32_t mode, int32_t quant,
+                         const float *sigma_row, const float *sigma_col, float sigma_tensor,
+                         uint64_t seed, uint32_t stream_id, int32_t L,
+                         uint8_t *bits, int32_t *T_out, uint8_t *sign_out);
+
 int32_t sco_encode(const float *X, int64_t rows, int64_t cols,
                    const int64_t *row_sel, int64_t nr, const int64_t *col_sel, int64_t nc,
                    int32_t tensor_id, int32_t mode,
@@ -224,6 +258,18 @@ int32_t sco_encode(const float *X, int64_t rows, int64_t cols,
                    uint64_t seed, uint32_t stream_id, int32_t L,
                    uint8_t *bits, int32_t *T_out, uint8_t *sign_out)
 {
+    return sco_encode_quant(X, rows, cols, row_sel, nr, col_sel, nc, tensor_id, mode, 0, sigma_row, sigma_col,
+                            sigma_tensor, seed, stream_id, L, bits, T_out, sign_out);
+}
+
+int32_t sco_encode_quant(const float *X, int64_t rows, int64_t cols,
+                         const int64_t *row_sel, int64_t nr, const int64_t *col_sel, int64_t nc,
+                         int32_t tensor_id, int32_t mode, int32_t quant,
+                         const float *sigma_row, const float *sigma_col, float sigma_tensor,
+                         uint64_t seed, uint32_t stream_id, int32_t L,
+                         uint8_t *bits, int32_t *T_out, uint8_t *sign_out)
+{
+    if (quant != 0 && quant != 1) return SCO_ERR_ARG;
     if (!X || !bits || L < 0 || nr < 0 || nc < 0) return SCO_ERR_ARG;
     for (int64_t a = 0; a < nr; ++a) { int64_t r = row_sel ? row_sel[a] : a; if (r < 0 || r >= rows) return SCO_ERR_ARG; }
     for (int64_t b = 0; b < nc; ++b) { int64_t c = col_sel ? col_sel[b] : b; if (c < 0 || c >= cols) return SCO_ERR_ARG; }
@@ -240,8 +286,9 @@ int32_t sco_encode(const float *X, int64_t rows, int64_t cols,
             float sigma = sigma_row ? sigma_row[r] : (sigma_col ? sigma_col[c] : sigma_tensor);
             float v = sco_normalise(x, sigma);
             int32_t sign = 0;
-            int32_t T = (mode == SCO_BIPOLAR_XNOR) ? sco_boundary_bipolar(v)
-                                                   : sco_boundary_unipolar(v, &sign);
+            int32_t T;
+            if (quant == 0) T = (mode == SCO_BIPOLAR_XNOR) ? sco_boundary_bipolar(v) : sco_boundary_unipolar(v, &sign);
+            else T = (mode == SCO_BIPOLAR_XNOR) ? sco_boundary_bipolar_int8(v) : sco_boundary_unipolar_int8(v, &sign);
             uint64_t elem = (uint64_t)r * (uint64_t)cols + (uint64_t)c;
             int64_t o = a * nc + b;
             if (T_out) T_out[o] = T;
@@ -439,7 +486,7 @@ int32_t sco_ladder_lengths(const float *g, int64_t M, int32_t group,
 
 
 /* ------------------------------------------------------------------------- */
-/* Sec. 3.3 (error tolerance): every exact output cell Y_ij is replaced by     */
+/* Sec. 3.2 (error tolerance): every exact output cell Y_ij is replaced by     */
 /* Y_ij (1 + alpha Z_ij), Z_ij independent standard normal, alpha a function   */
 /* of the stream length calibrated on measured SC error.  The paper's table of */
 /* alpha against L is, to its printed precision, alpha = coeff / L with        */

@@ -61,6 +61,10 @@ def _load():
     lib.sco_boundary_bipolar.restype = c.c_int32
     lib.sco_boundary_unipolar.argtypes = [c.c_float, i32p]
     lib.sco_boundary_unipolar.restype = c.c_int32
+    lib.sco_boundary_bipolar_int8.argtypes = [c.c_float]
+    lib.sco_boundary_bipolar_int8.restype = c.c_int32
+    lib.sco_boundary_unipolar_int8.argtypes = [c.c_float, i32p]
+    lib.sco_boundary_unipolar_int8.restype = c.c_int32
     lib.sco_random_byte.argtypes = [c.c_uint64, c.c_uint32, c.c_int32, c.c_uint64, c.c_int32]
     lib.sco_random_byte.restype = c.c_uint32
     lib.sco_stream_bit.argtypes = [c.c_uint64, c.c_uint32, c.c_int32, c.c_uint64, c.c_int32, c.c_int32]
@@ -76,6 +80,10 @@ def _load():
                                c.c_int32, c.c_int32, f32p, f32p, c.c_float,
                                c.c_uint64, c.c_uint32, c.c_int32, u8p, i32p, u8p]
     lib.sco_encode.restype = c.c_int32
+    lib.sco_encode_quant.argtypes = [f32p, c.c_int64, c.c_int64, i64p, c.c_int64, i64p, c.c_int64,
+                                     c.c_int32, c.c_int32, c.c_int32, f32p, f32p, c.c_float,
+                                     c.c_uint64, c.c_uint32, c.c_int32, u8p, i32p, u8p]
+    lib.sco_encode_quant.restype = c.c_int32
     lib.sco_gate_accumulate.argtypes = [c.c_int32, u8p, u8p, c.c_int32, u8p, u8p, c.c_int32,
                                         c.c_int64, c.c_int64, c.c_int64, i32p, i32p]
     lib.sco_gate_accumulate.restype = c.c_int32
@@ -149,6 +157,20 @@ def boundary_unipolar(v: float):
     return t, int(s.value)
 
 
+QUANT_DIRECT257, QUANT_INT8_THEN_257 = 0, 1
+
+
+def boundary_bipolar_int8(v: float) -> int:
+    """Sec. 4.2 two-step variant: int8 grid (q_max = 127) first, then the nearest of the 257 boundaries."""
+    return int(_load().sco_boundary_bipolar_int8(float(v)))
+
+
+def boundary_unipolar_int8(v: float):
+    s = ctypes.c_int32(0)
+    t = int(_load().sco_boundary_unipolar_int8(float(v), ctypes.byref(s)))
+    return t, int(s.value)
+
+
 def random_byte(seed: int, stream_id: int, tensor_id: int, elem: int, l: int) -> int:
     return int(_load().sco_random_byte(seed, stream_id, tensor_id, elem, l))
 
@@ -190,7 +212,7 @@ def row_absmax(X):
 
 
 def encode(X, tensor_id: int, mode: int, L: int, seed: int, stream_id: int = 0,
-           sigma_row=None, sigma_col=None, sigma_tensor: float = 1.0, row_sel=None, col_sel=None):
+           sigma_row=None, sigma_col=None, sigma_tensor: float = 1.0, row_sel=None, col_sel=None, quant: int = 0):
     """Streams of X[row_sel, col_sel]: returns (bits[nr, nc, L] uint8, T[nr, nc] int32, sign[nr, nc] uint8)."""
     X = _f32(X)
     rows, cols = X.shape
@@ -203,8 +225,8 @@ def encode(X, tensor_id: int, mode: int, L: int, seed: int, stream_id: int = 0,
     sign = np.zeros((nr, nc), dtype=np.uint8)
     sr = None if sigma_row is None else _f32(sigma_row)
     sc = None if sigma_col is None else _f32(sigma_col)
-    code = _load().sco_encode(_ptr(X, ctypes.c_float), rows, cols, _ptr(rs, ctypes.c_int64), nr,
-                              _ptr(cs, ctypes.c_int64), nc, tensor_id, mode,
+    code = _load().sco_encode_quant(_ptr(X, ctypes.c_float), rows, cols, _ptr(rs, ctypes.c_int64), nr,
+                              _ptr(cs, ctypes.c_int64), nc, tensor_id, mode, quant,
                               _ptr(sr, ctypes.c_float), _ptr(sc, ctypes.c_float), float(sigma_tensor),
                               seed, stream_id, L, _ptr(bits, ctypes.c_uint8), _ptr(T, ctypes.c_int32),
                               _ptr(sign, ctypes.c_uint8))
@@ -252,7 +274,7 @@ def expand_lengths(L_groups, M: int, group: int):
 
 
 def matmul(A, W, L_rows, mode: int, scale_a: int, scale_w: int, seed: int, stream_id: int = 0,
-           row_sel=None, col_sel=None):
+           row_sel=None, col_sel=None, quant: int = 0):
     """The whole path on the output entries (row_sel x col_sel): returns dict(P, C, sigma_a, sigma_w).
 
     ``L_rows`` has one entry per row of A (already expanded from groups).  Scales are always taken
@@ -271,8 +293,8 @@ def matmul(A, W, L_rows, mode: int, scale_a: int, scale_w: int, seed: int, strea
     sig_w = scales(W, scale_w, "col")
     Lsel = L_rows[rs]
     Lmax = int(Lsel.max()) if Lsel.size else 0
-    abits, _, asign = encode(A, 0, mode, Lmax, seed, stream_id, sigma_row=sig_a, row_sel=rs)
-    wbits, _, wsign = encode(W, 1, mode, Lmax, seed, stream_id, sigma_col=sig_w, col_sel=cs)
+    abits, _, asign = encode(A, 0, mode, Lmax, seed, stream_id, sigma_row=sig_a, row_sel=rs, quant=quant)
+    wbits, _, wsign = encode(W, 1, mode, Lmax, seed, stream_id, sigma_col=sig_w, col_sel=cs, quant=quant)
     P = gate_accumulate(mode, abits, asign, wbits, wsign, Lsel)
     C = decode(mode, P, K, Lsel, sig_a[rs], sig_w[cs])
     return {"P": P, "C": C, "sigma_a": sig_a, "sigma_w": sig_w}
@@ -307,7 +329,7 @@ def ladder_lengths(g, group: int, ladder, tau):
     return L
 
 
-SURROGATE_COEFF = 2.324    # alpha(L) = 2.324 / L reproduces the printed alpha column of Sec. 3.3's table
+SURROGATE_COEFF = 2.324    # alpha(L) = 2.324 / L reproduces the printed alpha column of Sec. 3.2's table
 
 
 def standard_normal(seed: int, stream_id: int, cell: int) -> float:
@@ -315,7 +337,7 @@ def standard_normal(seed: int, stream_id: int, cell: int) -> float:
 
 
 def surrogate_noise(Y, L_rows, coeff: float, seed: int, stream_id: int = 0):
-    """Sec. 3.3: Y (1 + (coeff / L_i) Z) with Z standard normal per output cell; rows with L = 0 give 0."""
+    """Sec. 3.2: Y (1 + (coeff / L_i) Z) with Z standard normal per output cell; rows with L = 0 give 0."""
     Y = _f32(Y)
     M, N = Y.shape
     L_rows = np.ascontiguousarray(L_rows, dtype=np.int32)
@@ -404,7 +426,8 @@ def scc(a: int, b: int, c: int, d: int) -> float:
     return float(_load().sco_scc(a, b, c, d))
 
 
-def matmul_cbsg(A, W, L_rows, scale_a: int, scale_w: int, seed: int, stream_id: int = 0, row_sel=None, col_sel=None):
+def matmul_cbsg(A, W, L_rows, scale_a: int, scale_w: int, seed: int, stream_id: int = 0, row_sel=None, col_sel=None,
+                quant: int = 0):
     """Bipolar SC product with the Sobol-8 / conditional-generation streams: dict(P, C, sigma_a, sigma_w)."""
     A, W = _f32(A), _f32(W)
     M, K = A.shape
@@ -415,8 +438,8 @@ def matmul_cbsg(A, W, L_rows, scale_a: int, scale_w: int, seed: int, stream_id: 
     cs = np.arange(N, dtype=np.int64) if col_sel is None else np.ascontiguousarray(col_sel, dtype=np.int64)
     sig_a = scales(A, scale_a, "row")
     sig_w = scales(W, scale_w, "col")
-    _, Ta, _ = encode(A, 0, BIPOLAR_XNOR, 0, seed, stream_id, sigma_row=sig_a, row_sel=rs)      # boundaries only
-    _, Tw, _ = encode(W, 1, BIPOLAR_XNOR, 0, seed, stream_id, sigma_col=sig_w, col_sel=cs)
+    _, Ta, _ = encode(A, 0, BIPOLAR_XNOR, 0, seed, stream_id, sigma_row=sig_a, row_sel=rs, quant=quant)   # boundaries only
+    _, Tw, _ = encode(W, 1, BIPOLAR_XNOR, 0, seed, stream_id, sigma_col=sig_w, col_sel=cs, quant=quant)
     Lsel = np.ascontiguousarray(L_rows[rs])
     P = np.zeros((rs.size, cs.size), dtype=np.int32)
     code = _load().sco_cbsg_gate_accumulate(_ptr(np.ascontiguousarray(Ta), ctypes.c_int32),

@@ -23,7 +23,7 @@ SC_L_CAP = 1024
 EXPORTS = (
     "sc_create", "sc_destroy", "sc_status_string", "sc_device_status", "sc_row_stats", "sc_assign_lengths",
     "sc_ladder_lengths", "sc_stream_bytes", "sc_encode", "sc_debug_unpack", "sc_workspace_bytes", "sc_matmul",
-    "sc_selftest_comparator", "sc_selftest_expansion", "sc_microbench", "sc_profile_enable", "sc_profile_read", "sc_launch_count",
+    "sc_selftest_comparator", "sc_selftest_expansion", "sc_selftest_bounded_wait", "sc_microbench", "sc_profile_enable", "sc_profile_read", "sc_launch_count",
     "sc_assign_lengths_static", "sc_weights_bytes", "sc_weights_prepare", "sc_weights_release",
     "sc_workspace_bytes_prepared", "sc_matmul_prepared", "sc_surrogate_noise",
     "sc_workspace_bytes_batched", "sc_matmul_batched", "sc_workspace_bytes_cbsg", "sc_matmul_cbsg", "sc_cbsg_scc",
@@ -95,6 +95,8 @@ def load():
     lib.sc_selftest_expansion.argtypes = []
     lib.sc_selftest_expansion.restype = i32
     lib.sc_microbench.argtypes = [vp, i32, i32, c.POINTER(c.c_float), c.POINTER(f64)]
+    lib.sc_selftest_bounded_wait.argtypes = [vp, i64, c.POINTER(i32), c.POINTER(i64)]
+    lib.sc_selftest_bounded_wait.restype = c.c_int
     lib.sc_profile_enable.argtypes = [vp, i32]
     lib.sc_profile_read.argtypes = [vp, c.POINTER(c.c_float)]
     lib.sc_launch_count.argtypes = [vp, c.POINTER(i64)]
@@ -270,6 +272,13 @@ def sc_selftest_comparator() -> int:
 
 def sc_selftest_expansion() -> int:
     return int(load().sc_selftest_expansion())
+
+
+def sc_selftest_bounded_wait(ctx, limit_cycles: int):
+    """Returns (site word, counter a, counter b), (clocks waited by the timed-out warp, by the aborted warp)."""
+    site, cyc = (ctypes.c_int32 * 3)(), (ctypes.c_int64 * 2)()
+    _check(load().sc_selftest_bounded_wait(ctx, int(limit_cycles), site, cyc), "sc_selftest_bounded_wait")
+    return tuple(int(x) for x in site), tuple(int(x) for x in cyc)
 
 
 def sc_microbench(ctx, kind: int, iters: int):

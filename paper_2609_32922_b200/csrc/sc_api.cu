@@ -750,29 +750,24 @@ int32_t sc_selftest_expansion(void)
     return mismatches;
 }
 
-sc_status sc_microbench(sc_ctx *ctx, int32_t kind, int32_t iters, float *ms_out, double *words_out)
+sc_status sc_selftest_bounded_wait(sc_ctx *ctx, int64_t limit_cycles, int32_t *site_host, int64_t *cycles_host)
 {
-    if (!ctx || !ms_out || !words_out || kind < 0 || kind > 4999999 || iters < 1) return SC_ERR_ARG;
+    if (!ctx || !site_host || !cycles_host || limit_cycles < 1 || limit_cycles > 2000000000LL) return SC_ERR_ARG;
     sc_ctx_impl *c = reinterpret_cast<sc_ctx_impl *>(ctx);
     if (cudaSetDevice(c->device) != cudaSuccess) return SC_ERR_CUDA;
-    if (kind >= 4000000) {      // accumulator / A-operand column placement probe: kind = 4000000 + 1000 * d_col + a_col
-        *words_out = 0.0;
-        const int d_col = (kind - 4000000) / 1000, a_col = (kind - 4000000) % 1000;
-        if (d_col + 192 > 512 || a_col + 64 > 512) return SC_ERR_ARG;
-        if (a_col + 64 > d_col && a_col < d_col + 192) return SC_ERR_ARG;      // operand would overlap the accumulator
-        return run_umma_interference(c, 0, 0, iters, ms_out, d_col, a_col) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
-    }
-    if (kind >= 2000000) {      // interference probe: kind = 2000000 + 100 * mode + n_side
-        *words_out = 0.0;
-        if ((kind - 2000000) / 100 > 8 || (kind - 2000000) % 100 > 24) return SC_ERR_ARG;
-        return run_umma_interference(c, (kind - 2000000) / 100, (kind - 2000000) % 100, iters, ms_out) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
-    }
-    if (kind >= 1000000) {      // side-latency probe: kind = 1000000 + 10 * mode + busy
-        *words_out = 0.0;
-        if ((kind - 1000000) / 10 > 4 || (kind - 1000000) % 10 > 1) return SC_ERR_ARG;
-        return run_umma_side_latency(c, (kind - 1000000) / 10, (kind - 1000000) % 10, iters, ms_out) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
-    }
-    if (kind >= 8) return run_umma_rate(c, kind - 8, iters, ms_out, words_out) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+    long long cyc[2] = {0, 0};
+    if (run_bounded_wait_selftest(c, (long long)limit_cycles, site_host, cyc) != cudaSuccess) return SC_ERR_CUDA;
+    cycles_host[0] = cyc[0];
+    cycles_host[1] = cyc[1];
+    return SC_OK;
+}
+
+sc_status sc_microbench(sc_ctx *ctx, int32_t kind, int32_t iters, float *ms_out, double *words_out)
+{
+    if (!ctx || !ms_out || !words_out || kind < 0 || kind > 9 || iters < 1 || iters > (1 << 22)) return SC_ERR_ARG;
+    sc_ctx_impl *c = reinterpret_cast<sc_ctx_impl *>(ctx);
+    if (cudaSetDevice(c->device) != cudaSuccess) return SC_ERR_CUDA;
+    if (kind >= 8) return run_mxf4_rate(c, kind == 8 ? 192 : 256, iters, ms_out, words_out) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
     return run_microbench(c, kind, iters, ms_out, words_out) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
 }
 

@@ -178,8 +178,11 @@ cudaError_t launch_assign_lengths(const float *g, int64_t M, int32_t group, doub
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    long long budget = llround(avg_budget * (double)M);
-    long long u = (long long)floor(avg_budget);
+    // a budget beyond Lmax per row means "every row at Lmax"; clamping first keeps the rounding in range for any
+    // finite budget
+    const double avg = fmin(avg_budget, (double)Lmax);
+    long long budget = llround(avg * (double)M);
+    long long u = (long long)floor(avg);
     u = u < Lmin ? Lmin : (u > Lmax ? Lmax : u);
     const int64_t ngroups = (M + group - 1) / group;
     const size_t use = ngroups <= kQCacheMax ? sizeof(uint32_t) * (size_t)ngroups : 0;

@@ -37,43 +37,25 @@
 
 namespace sc {
 
-#ifndef SC_A_GROUPS
-#define SC_A_GROUPS 3
-#endif
-#ifndef SC_W_GROUPS
-#define SC_W_GROUPS 3
-#endif
-#ifndef SC_ISSUERS
-#define SC_ISSUERS 2
-#endif
 constexpr int kUN = kTileNUmma;                // 192 output columns per tile
-#ifndef SC_RAW_UNITS
-#define SC_RAW_UNITS 3
-#endif
-constexpr int kRawUnits = SC_RAW_UNITS;        // plan units (kStagePlanes planes each) per TMA box / raw stage
+constexpr int kRawUnits = 3;                   // plan units (kStagePlanes planes each) per TMA box / raw stage
 constexpr int kRawPlanes = kRawUnits * kStagePlanes;
-#ifndef SC_RAW_STAGES
-#define SC_RAW_STAGES (SC_RAW_UNITS == 1 ? 3 : 2)
-#endif
-constexpr int kRawStages = SC_RAW_STAGES;
+constexpr int kRawStages = 2;
 constexpr int kOpSteps = 4;                    // MMA K-steps (32 bytes of K each) per operand stage
-#ifndef SC_OP_STAGES
-#define SC_OP_STAGES 4
-#endif
-constexpr int kOpStages = SC_OP_STAGES;
+constexpr int kOpStages = 4;
 constexpr int kEpiFirstWarp = 2, kEpiWarps = 4;
 // Expander warps work in groups; group g of a kind fills every groups-th operand stage.  An MMA issuer owns
 // fixed stages (a waiter that skipped a use of a stage could not tell the barrier's phases apart by parity;
 // the expanders, which may skip uses, wait on barriers that alternate between even and odd uses instead).
-constexpr int kAGroups = SC_A_GROUPS;          // activation expanders: groups of ...
+constexpr int kAGroups = 3;                    // activation expanders: groups of ...
 constexpr int kAFirstWarp = 6, kAWarps = 4;    // ... 4 warps (one per tensor-memory lane quarter)
-constexpr int kWGroups = SC_W_GROUPS;          // weight expanders: groups of ...
+constexpr int kWGroups = 3;                    // weight expanders: groups of ...
 constexpr int kWCols = 2;                      // (columns per W expander thread)
 constexpr int kWWarps = kTileNUmma / (32 * kWCols);   // ... 3 warps (64 columns each)
 constexpr int kFillWarps = kAWarps + kWWarps;  // arrivals per operand stage
 constexpr int kWFirstWarp = kAFirstWarp + kAGroups * kAWarps;
 constexpr int kAllExpWarps = kAGroups * kAWarps + kWGroups * kWWarps;
-constexpr int kIssuers = SC_ISSUERS;           // MMA issuer threads; issuer i owns the stages s with s % kIssuers == i
+constexpr int kIssuers = 2;                    // MMA issuer threads; issuer i owns the stages s with s % kIssuers == i
 constexpr int kIssuerBWarp = kAFirstWarp + kAllExpWarps;   // issuers 1.. live in the last warps
 constexpr int kUThreads = 32 * (kIssuerBWarp + kIssuers - 1);
 static_assert(kOpStages % kIssuers == 0, "an issuer must own fixed operand stages");
@@ -107,10 +89,7 @@ constexpr size_t kUmmaSmem = (size_t)kRawStages * kRawStageBytes + (size_t)kOpSt
 // four A stages fit.
 constexpr uint32_t kSfCols = 32;
 constexpr uint32_t kSfCol = kTmemCols - kSfCols;
-#ifndef SC_SINGLE_ACC_UNITS
-#define SC_SINGLE_ACC_UNITS 176
-#endif
-constexpr int32_t kSingleAccUnits = SC_SINGLE_ACC_UNITS;   // mean stage units per piece from which one accumulator is faster
+constexpr int32_t kSingleAccUnits = 176;   // mean stage units per piece from which one accumulator is faster
 static_assert(2 * kAccCols + 3 * kOpSteps * 8 + kSfCols <= kTmemCols && kAccCols + 4 * kOpSteps * 8 + kSfCols <= kTmemCols &&
               2 * kAccCols + 4 * kOpSteps * 8 <= kTmemCols && kOpStages >= 4, "tensor memory budget");
 
@@ -152,7 +131,8 @@ __device__ __forceinline__ bool u_mbar_try(uint32_t bar, uint32_t parity)
 // Bounded, abortable wait: false when the clock limit passes or another role has already given up.  The poll
 // loop itself is only the try_wait (a barrier operation costs ~100 cycles, and every cycle added to a poll is
 // added to the hand-over latency between roles); the abort flag and the clock are looked at every 64 polls.
-__device__ __forceinline__ bool u_mbar_wait(uint32_t bar, uint32_t parity, volatile int32_t *abort_flag)
+__device__ __forceinline__ bool u_mbar_wait(uint32_t bar, uint32_t parity, volatile int32_t *abort_flag,
+                                            long long limit_cycles = kUWaitCycles)
 {
     long long t0 = 0;
     for (uint32_t spins = 1;; ++spins) {
@@ -161,7 +141,7 @@ __device__ __forceinline__ bool u_mbar_wait(uint32_t bar, uint32_t parity, volat
             if (*abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kUWaitCycles) return false;
+            else if (now - t0 > limit_cycles) return false;
         }
     }
 }
@@ -170,6 +150,13 @@ __device__ __forceinline__ bool u_mbar_wait_warp(uint32_t bar, uint32_t parity, 
 {
     int ok = 1;
     if (lane == 0) ok = u_mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+}
+__device__ __forceinline__ bool u_mbar_wait_warp_limit(uint32_t bar, uint32_t parity, volatile int32_t *abort_flag, int lane,
+                                                       long long limit_cycles)
+{
+    int ok = 1;
+    if (lane == 0) ok = u_mbar_wait(bar, parity, abort_flag, limit_cycles) ? 1 : 0;
     return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
 }
 __device__ __forceinline__ void u_tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, uint32_t bar)
@@ -666,6 +653,60 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
         u_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
+}
+
+// ---- the bounded wait running out, on purpose ------------------------------------------------------------
+// One CTA, two warps, no tensor-core or TMA work: warp 0 waits with the core's own bounded wait on a barrier that
+// nobody ever arrives on, with a short limit; when the limit passes it records the wait site beside the status word
+// and raises the abort flag, exactly as a role of the core does.  Warp 1 waits on a second such barrier with the
+// default (long) limit and must leave through the abort flag.  The kernel then returns normally.
+constexpr int kSelftestWaitSite = 99;
+__global__ void __launch_bounds__(64)
+bounded_wait_selftest_kernel(long long limit_cycles, int32_t *scratch, long long *cycles_out)
+{
+    __shared__ uint64_t bars[2];
+    __shared__ int32_t s_abort_word;
+    volatile int32_t *s_abort = &s_abort_word;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        u_mbar_init(u_smem(&bars[0]), 1);
+        u_mbar_init(u_smem(&bars[1]), 1);
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const long long t0 = clock64();
+    bool ok;
+    if (warp == 0) {
+        ok = u_mbar_wait_warp_limit(u_smem(&bars[0]), 0u, s_abort, lane, limit_cycles);
+        if (!ok && lane == 0) {
+            if (atomicCAS(scratch + kSlotTimeoutSite, 0, kSelftestWaitSite | (warp << 8) | ((int)blockIdx.x << 16)) == 0) {
+                scratch[kSlotTimeoutSite + 1] = 1;
+                scratch[kSlotTimeoutSite + 2] = 2;
+            }
+            *s_abort = 1;
+            report(scratch + kSlotStatus, SC_ERR_TIMEOUT);
+        }
+    } else {
+        ok = u_mbar_wait_warp(u_smem(&bars[1]), 0u, s_abort, lane);      // leaves when warp 0 gives up
+    }
+    if (lane == 0) cycles_out[warp] = ok ? -1 : clock64() - t0;
+}
+
+cudaError_t run_bounded_wait_selftest(sc_ctx_impl *ctx, long long limit_cycles, int32_t site_out[3], long long cycles_out[2])
+{
+    long long *cyc = reinterpret_cast<long long *>(ctx->scratch + 1024);
+    cudaError_t e = cudaMemset(cyc, 0, 2 * sizeof(long long));
+    if (e != cudaSuccess) return e;
+    bounded_wait_selftest_kernel<<<1, 64>>>(limit_cycles, ctx->scratch, cyc);
+    count_launches(1);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return e;
+    e = cudaMemcpy(cycles_out, cyc, 2 * sizeof(long long), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return e;
+    return cudaMemcpy(site_out, ctx->scratch + kSlotTimeoutSite, 3 * sizeof(int32_t), cudaMemcpyDeviceToHost);
 }
 
 // ---- popcount corrections of the bipolar mode ---------------------------------------------------------

@@ -208,8 +208,7 @@ cudaError_t launch_surrogate(const float *Y, int64_t M, int64_t N, const int32_t
                              uint64_t seed, uint32_t stream_id, float *out, int32_t *status, cudaStream_t st);
 
 cudaError_t run_microbench(sc_ctx_impl *ctx, int kind, int iters, float *ms, double *words);
-cudaError_t run_umma_interference(sc_ctx_impl *ctx, int mode, int n_side, int n_mma, float *clk_per_mma, int d_col = 0, int a_col = 384);
-cudaError_t run_umma_side_latency(sc_ctx_impl *ctx, int mode, int busy, int iters, float *clk_per_iter);
-cudaError_t run_umma_rate(sc_ctx_impl *ctx, int variant, int iters, float *mclk, double *macs_per_sm);
+cudaError_t run_bounded_wait_selftest(sc_ctx_impl *ctx, long long limit_cycles, int32_t site_out[3], long long cycles_out[2]);
+cudaError_t run_mxf4_rate(sc_ctx_impl *ctx, int n_cols, int iters, float *mclk, double *macs_per_sm);
 
 }  // namespace sc

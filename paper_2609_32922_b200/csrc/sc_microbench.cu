@@ -1,6 +1,7 @@
-// Register-only instruction-mix loops: they measure the integer-pipe ceilings the GEMM core is bound by
-// (POPC, LOP3, IADD3 alone; the plain gate+popcount+add mix; the carry-save mix), so that the reported
-// roofline fraction has a measured denominator next to the nominal one.
+// Peak measurements for the roofline denominators.
+// Register-only instruction-mix loops measure the integer-pipe ceilings the ALU cores are bound by (POPC, LOP3, IADD3
+// alone; the plain gate+popcount+add mix; the carry-save mix); a bare chain of tcgen05.mma kind::mxf4 instructions
+// measures the issue-rate ceiling of the tensor-core core's instruction.
 #include "sc_device.cuh"
 #include "sc_internal.h"
 
@@ -142,6 +143,117 @@ cudaError_t run_microbench(sc_ctx_impl *ctx, int kind, int iters, float *ms, dou
     }
     count_launches(2);
     return cudaGetLastError();
+}
+
+
+// ---- issue rate of the tensor-core core's instruction --------------------------------------------------------------
+// One CTA per SM, one thread: a chain of `n_mma` block-scaled 4-bit MMAs (128 x n_cols x 64 each, A operand and scale
+// factors in tensor memory, B operand in shared memory, fp32 accumulators in tensor memory) on zero-filled operands,
+// eight per loop trip with precomputed descriptors, one commit at the end.  The elapsed SM clocks of the slowest SM
+// give multiply-accumulates per clock per SM.  The wait for the commit is bounded.
+__device__ __forceinline__ uint32_t mb_smem(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__global__ void __launch_bounds__(128, 1) mxf4_rate_kernel(int n_mma, int n_cols, long long *cycles_out)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    __shared__ uint32_t s_tmem;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kBytes = 8 * 256 * 32;                    // eight B tiles of up to 256 columns x 32 bytes of K
+    for (int i = threadIdx.x; i < kBytes / 4; i += blockDim.x) reinterpret_cast<uint32_t *>(smem)[i] = 0u;
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(mb_smem(&bar)) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(mb_smem(&s_tmem)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s_tmem;
+    {   // scale factors (columns 480..511): every byte 2^0; A operand (columns 256..319): zeros
+        uint32_t v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[k] = 0x7F7F7F7Fu;
+        const uint32_t lane_base = ((uint32_t)warp * 32u) << 16;
+        for (uint32_t c = 480; c < 512; c += 8)
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                         ::"r"(tmem + c + lane_base), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+        for (uint32_t c = 256; c < 320; c += 8)
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1};" ::"r"(tmem + c + lane_base), "r"(0u) : "memory");
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (warp == 0 && lane == 0) {
+        const uint32_t lbo = (uint32_t)n_cols * 16u;        // bytes between the two 16-byte K chunks of a tile
+        uint64_t bd[8];
+        uint32_t ad[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t addr = mb_smem(smem) + (uint32_t)k * (uint32_t)n_cols * 32u;
+            bd[k] = (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
+                    ((uint64_t)(128u >> 4) << 32) | (1ull << 46);
+            ad[k] = tmem + 256u + (uint32_t)k * 8u;
+        }
+        // kind::mxf4: e2m1 x e2m1, K-major, ue8m0 scale factors, M = 128
+        const uint32_t idesc = (1u << 7) | (1u << 10) | ((uint32_t)(n_cols >> 3) << 17) | (1u << 23) | (8u << 24);
+        const long long t0 = clock64();
+        for (int g0 = 0; g0 < n_mma; g0 += 8) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                             "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], [%1], %2, %3, [%5], [%6], p;\n\t}"
+                             ::"r"(tmem), "r"(ad[k]), "l"(bd[k]), "r"(idesc), "r"((uint32_t)((g0 | k) != 0)), "r"(tmem + 480u),
+                               "r"(tmem + 496u) : "memory");
+        }
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mb_smem(&bar)) : "memory");
+        uint32_t ok = 0;
+        const long long limit = t0 + 4000000000LL;
+        while (!ok && clock64() < limit)
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(ok) : "r"(mb_smem(&bar)) : "memory");
+        cycles_out[blockIdx.x] = ok ? (clock64() - t0) : -1;
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+    }
+}
+
+// *mclk = SM clocks of the slowest SM / 1e6; *macs = multiply-accumulates per SM.
+cudaError_t run_mxf4_rate(sc_ctx_impl *ctx, int n_cols, int iters, float *mclk, double *macs)
+{
+    iters = (iters + 7) / 8 * 8;
+    long long *cyc = reinterpret_cast<long long *>(ctx->scratch + 1024);
+    const size_t smem = 8 * 256 * 32;
+    cudaError_t e = cudaFuncSetAttribute(mxf4_rate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaMemset(cyc, 0, sizeof(long long) * 256);
+    if (e != cudaSuccess) return e;
+    mxf4_rate_kernel<<<ctx->sm_count, 128, smem>>>(iters, n_cols, cyc);
+    count_launches(1);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return e;
+    long long host[256];
+    e = cudaMemcpy(host, cyc, sizeof(long long) * 256, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return e;
+    long long worst = 0;
+    for (int i = 0; i < ctx->sm_count && i < 256; ++i) {
+        if (host[i] <= 0) return cudaErrorLaunchTimeout;
+        if (host[i] > worst) worst = host[i];
+    }
+    *mclk = (float)((double)worst / 1.0e6);
+    *macs = 128.0 * n_cols * 64.0 * (double)iters;
+    return cudaSuccess;
 }
 
 }  // namespace sc

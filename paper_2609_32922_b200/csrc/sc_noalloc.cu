@@ -19,7 +19,7 @@
 namespace sc {
 
 constexpr int kStaticThreads = 1024;
-constexpr int kStaticHeaderWords = 64;                        // 256 bytes: [0] status, [2..3] total length
+constexpr int kStaticHeaderWords = 64;                        // 256 bytes: word [0] is the status of the call, the rest is unused
 
 // File-scope scratch: one grid value per group plus the header.  Every GPU that loads the library holds
 // these SC_STATIC_MAX_GROUPS * 4 + 256 bytes (about 1 MB) until the process exits.
@@ -77,7 +77,7 @@ assign_lengths_static_kernel(const float *__restrict__ g, int64_t M, int32_t gro
     int32_t *status = reinterpret_cast<int32_t *>(scratch);
     const int64_t ngroups = (M + group - 1) / group;
 
-    if (threadIdx.x == 0) { scratch[0] = 0u; scratch[2] = 0u; scratch[3] = 0u; }   // header starts at zero
+    if (threadIdx.x == 0) scratch[0] = 0u;                   // the status word starts at zero
     __syncthreads();
 
     float lo_f = INFINITY, hi_f = -INFINITY;
@@ -176,8 +176,11 @@ extern "C" sc_status sc_assign_lengths_static(const float *g, int64_t M, int32_t
     if (Lmin < 0 || Lmax < Lmin || Lmax > SC_L_CAP) return SC_ERR_LENGTH;
     uint32_t *scratch = nullptr;
     if (static_scratch_address(&scratch) != cudaSuccess) return SC_ERR_CUDA;
-    const long long budget = llround(avg_budget * (double)M);
-    long long u = (long long)floor(avg_budget);
+    // a budget beyond Lmax per row means "every row at Lmax"; clamping first keeps the rounding in range for any
+    // finite budget
+    const double avg = fmin(avg_budget, (double)Lmax);
+    const long long budget = llround(avg * (double)M);
+    long long u = (long long)floor(avg);
     u = u < Lmin ? Lmin : (u > Lmax ? Lmax : u);
     assign_lengths_static_kernel<<<1, kStaticThreads, 0, (cudaStream_t)stream>>>(
         g, M, group, budget, (int32_t)u, Lmin, Lmax, L_out, scratch, status_out,

@@ -1,4 +1,4 @@
-// Gaussian-perturbed surrogate of an SC product (Sec. 3.3, error tolerance): out_ij = Y_ij (1 + alpha(L_i) Z_ij),
+// Gaussian-perturbed surrogate of an SC product (Sec. 3.2, error tolerance): out_ij = Y_ij (1 + alpha(L_i) Z_ij),
 // Z_ij independent standard normal, alpha(L) = coeff / L (the paper's table of alpha against L is coeff = 2.324 to
 // its printed precision).  A cheap stand-in for the stochastic matmul in model-level sweeps: one pass over Y, HBM-bound.
 //
@@ -23,17 +23,19 @@ __device__ __forceinline__ double standard_normal(const PhiloxKeys &ks, uint32_t
 }
 
 __global__ void __launch_bounds__(256)
-surrogate_kernel(const __grid_constant__ PhiloxKeys ks, const float *__restrict__ Y, int64_t M, int64_t N,
+surrogate_kernel(const __grid_constant__ PhiloxKeys ks, const float *Y, int64_t M, int64_t N,
                  const int32_t *__restrict__ L, int32_t group, double coeff, uint32_t stream_word,
-                 float *__restrict__ out, int32_t *status)
+                 float *out, int32_t *status)
 {
+    // `out` may be the same buffer as `Y` (each thread reads a cell before it writes it): neither pointer is
+    // declared restrict and Y is read with plain (coherent) loads.
     bool bad_value = false, bad_length = false;
     for (int64_t i = blockIdx.y; i < M; i += gridDim.y) {
         int32_t len = L ? __ldg(L + i / group) : 1;
         if (len < 0) { bad_length = true; len = 0; }
         const double alpha = len > 0 ? coeff / (double)len : 0.0;
         for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < N; j += (int64_t)gridDim.x * blockDim.x) {
-            float y = __ldg(Y + i * N + j);
+            float y = Y[i * N + j];
             if (is_nonfinite(y)) { bad_value = true; y = 0.0f; }
             float r = 0.0f;
             if (len > 0) r = (float)((double)y * (1.0 + alpha * standard_normal(ks, stream_word, (uint64_t)(i * N + j))));

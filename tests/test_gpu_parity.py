@@ -207,12 +207,21 @@ def test_config4_dit_grouped_sampled(sc, binding, oracle, core):
     _sampled_parity(sc, binding, oracle, w, A, W, L_groups, 512, 8, 12, 24, core=core)
 
 
-@pytest.mark.parametrize("core", [0, 4])
-@pytest.mark.parametrize("which,L", [(0, 32), (1, 1023), (2, 8), (3, 32), (3, 128)])
-def test_config5_vit_l_sweep_sampled(sc, binding, oracle, which, L, core):
+@pytest.mark.parametrize("L", [8, 32, 128, 512, 1023])
+@pytest.mark.parametrize("which", [0, 1, 2, 3])        # qkv, proj, fc1 (bipolar), fc2 (unipolar)
+def test_config5_vit_l_sweep_sampled(sc, binding, oracle, which, L):
+    """All twenty (layer shape, L) cells of the ViT-L/14 sweep at full size with the default core, each on sampled
+    rows x columns evaluated by the oracle."""
     w = wl.vit_l_layers(L)[which]
     A, W = wl.make_inputs(w)
-    _sampled_parity(sc, binding, oracle, w, A, W, None, L, 1, 8, 16, core=core)
+    _sampled_parity(sc, binding, oracle, w, A, W, None, L, 1, 8, 16, core=0)
+
+
+@pytest.mark.parametrize("which,L", [(1, 32), (3, 128)])
+def test_config5_cells_on_the_integer_core(sc, binding, oracle, which, L):
+    w = wl.vit_l_layers(L)[which]
+    A, W = wl.make_inputs(w)
+    _sampled_parity(sc, binding, oracle, w, A, W, None, L, 1, 8, 16, core=2)
 
 
 def test_row_independence_and_prefix_on_gpu(sc, binding):
@@ -259,6 +268,31 @@ def test_device_detected_errors(sc, binding):
     with pytest.raises(binding.ScError) as e:
         binding.sc_matmul(sc.ctx, dA, dW, None, 2000, p, None, C, ws)
     assert e.value.code == binding.SC_ERR_LENGTH
+
+
+def test_bounded_wait_runs_out_and_the_context_survives(sc, binding, oracle):
+    """Failure detection without a fault: a wait of the tensor-core core's own wait routine on a barrier that is never
+    signalled gives up after its (here short) clock limit, records SC_ERR_TIMEOUT and the wait site, the second role
+    leaves through the abort flag, the kernel returns within milliseconds and the next product is bit-exact."""
+    import time
+    limit = 1_000_000                                             # SM clocks: about half a millisecond
+    binding.sc_selftest_bounded_wait(sc.ctx, 1000)                # first launch loads the kernel's code
+    assert sc.device_status() == binding.SC_ERR_TIMEOUT
+    t0 = time.perf_counter()
+    site, cycles = binding.sc_selftest_bounded_wait(sc.ctx, limit)
+    seconds = time.perf_counter() - t0
+    assert site[0] & 0xFF == 99 and (site[0] >> 8) & 0xFF == 0 and site[0] >> 16 == 0 and site[1:] == (1, 2)
+    assert limit < cycles[0] < 20 * limit                         # gave up after the limit, not much later
+    assert 0 < cycles[1] < 30 * limit                             # the other role left through the abort flag
+    assert seconds < 0.5
+    assert sc.device_status() == binding.SC_ERR_TIMEOUT
+    assert sc.device_status() == 0                                # cleared by the read, site slots too
+    w, L_rows = wl.small_ragged(seed=11, mode="bipolar")
+    A, W = wl.make_inputs(w)
+    P, C = T.gpu_matmul(sc, binding, w, A, W, L_rows, 100, core=4)
+    ref = T.oracle_matmul(oracle, w, A, W, L_rows)
+    assert np.array_equal(P, ref["P"]) and T.close_enough(C, ref["C"])
+    assert sc.device_status() == 0
 
 
 @pytest.mark.parametrize("core", [0, 4])

@@ -1,4 +1,4 @@
-"""GPU parity of the Gaussian surrogate (Sec. 3.3) against the oracle on the same seeded inputs.
+"""GPU parity of the Gaussian surrogate (Sec. 3.2) against the oracle on the same seeded inputs.
 Tolerance: the kernel evaluates the multiplier 1 + alpha Z in binary64 like the oracle (device log / cos / sqrt are
 within a few binary64 ulps of the host's), so after rounding to binary32 the two agree to 1e-6 relative / 1e-7
 absolute, the tolerance of the decoded outputs of the main path."""

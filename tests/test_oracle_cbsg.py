@@ -3,7 +3,7 @@
 The cycle-by-cycle multiplier is checked against: the structure of the Sobol sequences (permutations, stratified
 prefixes, the joint net of dimensions 1 and 2), a closed form of the XNOR count written here from cumulative counts,
 exactness at full length for boundaries on coarse grids (an 8-bit operand is recovered exactly at L = 256, Sec. 3.2),
-zero cross-correlation there (Appendix A.1), and an error that falls like 1/L rather than 1/sqrt(L) (Sec. 3.3's table).
+zero cross-correlation there (Appendix A.1), and an error that falls like 1/L rather than 1/sqrt(L) (Sec. 3.2's table).
 The match with the authors' own kernel cannot be checked: parity unpinned."""
 import numpy as np
 
@@ -83,9 +83,30 @@ def test_exact_products_and_zero_correlation_on_coarse_grids(oracle):
     assert oracle.scc(100, 0, 0, 156) == 1.0 and oracle.scc(0, 100, 156, 0) == -1.0
 
 
+def test_scc_piecewise_definition_hand_worked(oracle):
+    """Appendix A.1's two-case normalisation, worked by hand (a, b, c, d = cycles with the bit pair 11, 10, 01, 00).
+    Negative branch with a > d, where the max(a - d, 0) term matters:
+      (50, 30, 20, 0): ad - bc = -600, D = 80 * 70 - 100 * 50 = 600            -> -1 (as anti-correlated as the marginals allow)
+      (40, 30, 20, 10): ad - bc = -200, D = 70 * 60 - 100 * 30 = 1200          -> -1/6 (without the max term: -200/4200)
+    Negative branch with a <= d (the term vanishes): (5, 30, 20, 45): (225 - 600) / (35 * 25) = -3/7.
+    Positive branch: (40, 10, 20, 30): ad - bc = 1000, D = 100 * min(50, 60) - 50 * 60 = 2000 -> 1/2;
+    with the roles of the marginals swapped, (40, 20, 10, 30): D = 100 * 50 - 60 * 50 = 2000 -> 1/2.
+    Independent pair counts (ad = bc) give 0 in either branch."""
+    assert oracle.scc(50, 30, 20, 0) == -1.0
+    assert abs(oracle.scc(40, 30, 20, 10) - (-1.0 / 6.0)) < 1e-15
+    assert abs(oracle.scc(5, 30, 20, 45) - (-3.0 / 7.0)) < 1e-15
+    assert oracle.scc(40, 10, 20, 30) == 0.5 and oracle.scc(40, 20, 10, 30) == 0.5
+    assert oracle.scc(20, 20, 30, 30) == 0.0 and oracle.scc(0, 0, 0, 0) == 0.0
+    # bounded by 1 in magnitude over every table with L = 12
+    for a in range(13):
+        for b in range(13 - a):
+            for c in range(13 - a - b):
+                assert -1.0 - 1e-12 <= oracle.scc(a, b, c, 12 - a - b - c) <= 1.0 + 1e-12
+
+
 def test_error_falls_like_one_over_L(oracle):
     """Root-mean-square error of the decoded pair product over random boundaries: error x L stays within a band
-    (decay like 1/L, the law of Sec. 3.3's table, whose alpha x L is 2.32), far below the sqrt((1 - (a w)^2) / L) of
+    (decay like 1/L, the law of Sec. 3.2's table, whose alpha x L is 2.32), far below the sqrt((1 - (a w)^2) / L) of
     independent streams at the same length."""
     rng = np.random.default_rng(3)
     pairs = [(int(rng.integers(0, 257)), int(rng.integers(0, 257))) for _ in range(400)]

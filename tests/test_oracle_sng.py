@@ -191,3 +191,53 @@ def test_scales(oracle):
     with pytest.raises(oracle.OracleError) as e:
         oracle.scales(bad, oracle.SCALE_PER_ROW, "row")
     assert e.value.code == oracle.ERR_NONFINITE
+
+
+def test_int8_two_step_boundaries(oracle):
+    """Sec. 4.2's fused quantisation: the int8 grid (q_max = 127, Sec. 3.1) first, then one of the 257 boundaries.
+    Fixed by the text: the grid has 255 points, -1 / 0 / +1 are grid points, and the bipolar stream probability of a
+    grid point is (x_hat + q_max) / (2 q_max) (Sec. 3.1), so the boundary is the one nearest to 256 times that."""
+    from fractions import Fraction
+    assert oracle.boundary_bipolar_int8(-1.0) == 0
+    assert oracle.boundary_bipolar_int8(0.0) == 128
+    assert oracle.boundary_bipolar_int8(1.0) == 256
+    levels = []
+    for q in range(-127, 128):
+        T = oracle.boundary_bipolar_int8(q / 127.0)
+        target = Fraction(q + 127, 254) * 256                      # exact position of the grid point on the 0..256 scale
+        assert abs(T - target) < Fraction(1, 2)                    # nearest boundary; never a tie (127 is odd)
+        levels.append(T)
+    assert levels == sorted(levels) and len(set(levels)) == 255    # monotone, the 255 grid points stay distinct
+    assert set(range(257)) - set(levels) == {64, 192}              # two of the 257 boundaries are never used
+    # values between grid points snap to the grid first (round half to even in binary32), e.g. 0.004 -> x_hat = 1
+    assert oracle.boundary_bipolar_int8(0.004) == oracle.boundary_bipolar_int8(1 / 127.0) == 129
+    assert oracle.boundary_bipolar_int8(0.0039) == 128             # 127 * 0.0039 = 0.4953 -> 0
+    xs = np.linspace(-1, 1, 4001)
+    Ts = [oracle.boundary_bipolar_int8(float(x)) for x in xs]
+    assert Ts == sorted(Ts)
+    assert max(abs(T / 128.0 - 1.0 - x) for T, x in zip(Ts, xs)) <= 1 / 254 + 1 / 256 + 1e-6   # half a grid step + half a boundary step
+    # unipolar: sign and magnitude, magnitude grid 0..127 -> boundary nearest to 256 |x_hat| / 127
+    assert oracle.boundary_unipolar_int8(0.0) == (0, 0)
+    assert oracle.boundary_unipolar_int8(1.0) == (256, 0) and oracle.boundary_unipolar_int8(-1.0) == (256, 1)
+    mags = []
+    for q in range(128):
+        T, s = oracle.boundary_unipolar_int8(-q / 127.0)
+        assert s == (1 if q else 0) and abs(T - Fraction(q, 127) * 256) < Fraction(1, 2)
+        mags.append(T)
+    assert mags == sorted(mags) and len(set(mags)) == 128
+
+
+def test_int8_variant_changes_only_the_boundary(oracle):
+    """Streams of the two-step variant are the comparator outputs of its own boundaries on the same draws."""
+    rng = np.random.default_rng(2)
+    X = rng.uniform(-1, 1, size=(5, 9)).astype(np.float32)
+    for mode in (0, 1):
+        b0, T0, s0 = oracle.encode(X, 0, mode, 40, seed=9, stream_id=2)
+        b1, T1, s1 = oracle.encode(X, 0, mode, 40, seed=9, stream_id=2, quant=oracle.QUANT_INT8_THEN_257)
+        assert np.array_equal(s0, s1) and not np.array_equal(T0, T1) and np.abs(T0 - T1).max() <= 2
+        for i in range(5):
+            for d in range(9):
+                want = oracle.boundary_bipolar_int8(float(X[i, d])) if mode == 0 else oracle.boundary_unipolar_int8(float(X[i, d]))[0]
+                assert T1[i, d] == want
+                for l in range(40):
+                    assert b1[i, d, l] == (1 if oracle.random_byte(9, 2, 0, i * 9 + d, l) < want else 0)

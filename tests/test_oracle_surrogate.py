@@ -1,4 +1,4 @@
-"""Pins of the oracle's Gaussian surrogate (Sec. 3.3): the noise scale against the paper's printed table,
+"""Pins of the oracle's Gaussian surrogate (Sec. 3.2): the noise scale against the paper's printed table,
 the normal variates against the moments and the distribution function of N(0, 1), and the algebra of the output."""
 import math
 import os

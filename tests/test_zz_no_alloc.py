@@ -57,3 +57,44 @@ def test_static_assign_matches_context_based_entry_point_twice():
     assert rc == b.SC_ERR_SHAPE
     assert sc.device_status() == 0
     sc.close()
+
+
+def test_static_assign_at_its_limits():
+    """The largest size the fixed array holds (the last group short), a budget that saturates every row -- however large,
+    as long as it is finite -- and a non-finite metric: lengths, total and status must equal the context-based call's."""
+    import torch
+    from paper_2609_32922_b200 import build, binding as b
+    build.build()
+    torch.cuda.set_device(0)
+    sc = b.ScGemm(0)
+    rng = np.random.default_rng(321)
+    group = 2
+    M = b.SC_STATIC_MAX_GROUPS * group - 1                 # ceil(M / group) == SC_STATIC_MAX_GROUPS, last group of one row
+    g_host = np.abs(rng.standard_normal(M)).astype(np.float32)
+    g = torch.from_numpy(g_host).cuda()
+    n = (M + group - 1) // group
+    assert n == b.SC_STATIC_MAX_GROUPS
+    for avg, Lmin, Lmax in ((40.0, 4, 300), (1024.0, 4, 300), (1e300, 4, 300)):
+        L_ref, realised = sc.assign_lengths(g, group, avg, Lmin, Lmax, want_realized=True)
+        assert sc.device_status() == 0
+        L = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+        total = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+        b.sc_assign_lengths_static(g, group, avg, Lmin, Lmax, L, status, total)
+        torch.cuda.synchronize()
+        assert torch.equal(L, L_ref)
+        assert int(status.item()) == b.SC_OK and int(total.item()) == round(realised * M)
+        if avg >= Lmax:
+            assert (L == Lmax).all() and int(total.item()) == Lmax * M
+    # a non-finite metric is treated as 0 and reported; lengths still equal the context-based call's
+    g_bad = g.clone()
+    g_bad[12345] = float("nan")
+    L_ref = sc.assign_lengths(g_bad, group, 40.0, 4, 300)
+    assert sc.device_status() == b.SC_ERR_NONFINITE
+    L = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+    status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    b.sc_assign_lengths_static(g_bad, group, 40.0, 4, 300, L, status, None)
+    torch.cuda.synchronize()
+    assert torch.equal(L, L_ref) and int(status.item()) == b.SC_ERR_NONFINITE
+    assert sc.device_status() == 0                          # the static call never touches a context's status word
+    sc.close()
