@@ -44,6 +44,11 @@ FP4_TO_BF16_NOMINAL = 4.0       # dense tensor peaks: 9 PFLOP/s fp4 vs 2.25 PFLO
 # retires 32 stream bit-ops; 148 SMs at the maximum SM clock.
 POPC_PER_CLK_PER_SM = 16
 
+# Beside the headline workload the default run times these for a few steps each (kernels launched one by one): the
+# per-row mixed-precision configuration, the grouped DiT-like one, and the widest bipolar and the unipolar layer of the
+# ViT-L/14 sweep at L = 128.
+OTHER_CONFIGS = ("vit_b16_qkv_mixed", "dit_xl2_linear_grouped", "vit_l14_fc1_L128", "vit_l14_fc2_L128")
+
 
 def parse_args():
     ap = argparse.ArgumentParser()
@@ -58,6 +63,7 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="launch the step's kernels one by one instead of replaying "
                                                             "a CUDA graph captured from the same calls")
     ap.add_argument("--microbench", action="store_true", help="also report measured integer-pipe peaks")
+    ap.add_argument("--no-configs", action="store_true", help="skip the short runs of the other benchmark configurations")
     ap.add_argument("--sweep", metavar="FILE", help="time every benchmark configuration (all five configs, every "
                     "L of the ViT-L sweep) and write a table to FILE instead of the JSON line")
     ap.add_argument("--attention", metavar="FILE", help="time the batched attention products (qk and av per head, "
@@ -210,9 +216,79 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def measure_workload(sc, dev, name, core, reps=None):
+    """One workload through the public calls, kernels launched one by one: the whole step (min of `reps` runs, CUDA events
+    on the launching stream), the core phase from the library's own phase events, and the same step with prepared weights.
+    Operands of every workload here exceed the L2 capacity together with their stream planes, or are flushed by the
+    next workload's allocation; the headline line of the default run flushes L2 explicitly instead."""
+    import torch
+    from paper_2609_32922_b200 import binding, workloads as wl
+    w = get_workload(name)
+    A_h, W_h = wl.make_inputs(w)
+    A, W = torch.from_numpy(A_h).to(dev), torch.from_numpy(W_h).to(dev)
+    if w.policy:
+        avg, Lmin, Lmax, group = w.policy
+    else:
+        avg, Lmin, Lmax, group = float(w.uniform_L), min(8, w.uniform_L), w.uniform_L, 1
+    params = binding.make_params(mode=MODES[w.mode], scale_a=SCALES[w.scale_a], scale_w=SCALES[w.scale_w],
+                                 group=group, seed=w.seed, core=core)
+    g = torch.empty(w.M, dtype=torch.float32, device=dev)
+    L = torch.empty((w.M + group - 1) // group, dtype=torch.int32, device=dev)
+    C = torch.empty((w.M, w.N), dtype=torch.float32, device=dev)
+    ws = sc.workspace(binding.sc_workspace_bytes(w.M, w.K, w.N, Lmax, params))
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+
+    def step():
+        binding.sc_row_stats(sc.ctx, A, g)
+        binding.sc_assign_lengths(sc.ctx, g, group, avg, Lmin, Lmax, L)
+        binding.sc_matmul(sc.ctx, A, W, L, Lmax, params, None, C, ws)
+
+    if reps is None:
+        reps = 3 if w.M * w.N * w.K * Lmax < 2e13 else 1
+    for _ in range(2 if reps > 1 else 1):
+        step()
+    torch.cuda.synchronize()
+    binding.sc_profile_enable(sc.ctx, True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    step_ms, core_ms = [], []
+    for _ in range(reps):
+        flush.zero_()
+        e0.record()
+        step()
+        e1.record()
+        torch.cuda.synchronize()
+        step_ms.append(e0.elapsed_time(e1))
+        core_ms.append(binding.sc_profile_read(sc.ctx)["core"])
+    binding.sc_profile_enable(sc.ctx, False)
+    # the same step with the W side prepared once (static weights)
+    prepared = sc.prepare_weights(W, Lmax, params)
+
+    def step_prepared():
+        binding.sc_row_stats(sc.ctx, A, g)
+        binding.sc_assign_lengths(sc.ctx, g, group, avg, Lmin, Lmax, L)
+        binding.sc_matmul_prepared(sc.ctx, A, prepared[0], L, Lmax, params, None, C, ws)
+
+    step_prepared()
+    prep_ms = []
+    for _ in range(reps):
+        flush.zero_()
+        e0.record()
+        step_prepared()
+        e1.record()
+        torch.cuda.synchronize()
+        prep_ms.append(e0.elapsed_time(e1))
+    binding.sc_weights_release(prepared[0])
+    sum_L = float(oracle_free_sum_lengths(L, group, w.M))
+    bitops = float(w.N) * w.K * sum_L
+    out = {"workload": name, "M": w.M, "K": w.K, "N": w.N, "mode": w.mode, "mean_L": sum_L / w.M, "bitops": bitops,
+           "step_ms": min(step_ms), "core_ms": min(core_ms), "prepared_step_ms": min(prep_ms), "reps": reps,
+           "tensor_core": core in (0, 4) and w.K * Lmax <= (1 << 24)}
+    del A, W, C, prepared, ws, flush
+    return out
+
+
 def run_sweep(args):
     """Every configuration once: whole-step and core-only throughput, written as a markdown table."""
-    import numpy as np
     import torch
     from paper_2609_32922_b200 import binding, build, workloads as wl
     build.build()
@@ -227,63 +303,11 @@ def run_sweep(args):
         names += [w.name for w in wl.vit_l_layers(L)]
     rows = []
     for name in names:
-        w = get_workload(name)
-        A_h, W_h = wl.make_inputs(w)
-        A, W = torch.from_numpy(A_h).to(dev), torch.from_numpy(W_h).to(dev)
-        if w.policy:
-            avg, Lmin, Lmax, group = w.policy
-        else:
-            avg, Lmin, Lmax, group = float(w.uniform_L), min(8, w.uniform_L), w.uniform_L, 1
-        params = binding.make_params(mode=MODES[w.mode], scale_a=SCALES[w.scale_a], scale_w=SCALES[w.scale_w],
-                                     group=group, seed=w.seed, core=args.core)
-        g = torch.empty(w.M, dtype=torch.float32, device=dev)
-        L = torch.empty((w.M + group - 1) // group, dtype=torch.int32, device=dev)
-        C = torch.empty((w.M, w.N), dtype=torch.float32, device=dev)
-        ws = sc.workspace(binding.sc_workspace_bytes(w.M, w.K, w.N, Lmax, params))
-
-        def step():
-            binding.sc_row_stats(sc.ctx, A, g)
-            binding.sc_assign_lengths(sc.ctx, g, group, avg, Lmin, Lmax, L)
-            binding.sc_matmul(sc.ctx, A, W, L, Lmax, params, None, C, ws)
-
-        reps = 3 if w.M * w.N * w.K * Lmax < 2e13 else 1
-        for _ in range(2 if reps > 1 else 1):
-            step()
-        torch.cuda.synchronize()
-        binding.sc_profile_enable(sc.ctx, True)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        step_ms, core_ms = [], []
-        for _ in range(reps):
-            e0.record()
-            step()
-            e1.record()
-            torch.cuda.synchronize()
-            step_ms.append(e0.elapsed_time(e1))
-            core_ms.append(binding.sc_profile_read(sc.ctx)["core"])
-        binding.sc_profile_enable(sc.ctx, False)
-        # the same step with the W side prepared once (static weights)
-        prepared = sc.prepare_weights(W, Lmax, params)
-
-        def step_prepared():
-            binding.sc_row_stats(sc.ctx, A, g)
-            binding.sc_assign_lengths(sc.ctx, g, group, avg, Lmin, Lmax, L)
-            binding.sc_matmul_prepared(sc.ctx, A, prepared[0], L, Lmax, params, None, C, ws)
-
-        step_prepared()
-        prep_ms = []
-        for _ in range(reps):
-            e0.record()
-            step_prepared()
-            e1.record()
-            torch.cuda.synchronize()
-            prep_ms.append(e0.elapsed_time(e1))
-        binding.sc_weights_release(prepared[0])
-        sum_L = float(oracle_free_sum_lengths(L, group, w.M))
-        bitops = float(w.N) * w.K * sum_L
-        t, tc, tp = min(step_ms) * 1e-3, min(core_ms) * 1e-3, min(prep_ms) * 1e-3
-        rows.append((name, w.M, w.K, w.N, w.mode, sum_L / w.M, bitops, t * 1e3, bitops / t, float(w.M) * w.N * w.K / t,
-                     tc * 1e3, bitops / tc, bitops / tc / alu_peak, tp * 1e3, bitops / tp))
-        del A, W, C, prepared
+        m = measure_workload(sc, dev, name, args.core)
+        t, tc, tp, bitops = m["step_ms"] * 1e-3, m["core_ms"] * 1e-3, m["prepared_step_ms"] * 1e-3, m["bitops"]
+        rows.append((name, m["M"], m["K"], m["N"], m["mode"], m["mean_L"], bitops, t * 1e3, bitops / t,
+                     float(m["M"]) * m["N"] * m["K"] / t, tc * 1e3, bitops / tc, bitops / tc / alu_peak, tp * 1e3,
+                     bitops / tp))
     assert sc.device_status() == 0
     with open(args.sweep, "w") as f:
         f.write("| workload | M | K | N | mode | mean L | bit-ops | step ms | step bit-op/s | equiv MAC/s | core ms | "
@@ -637,21 +661,33 @@ def main():
     uses_tensor = args.core in (0, 4) and w.K * Lmax <= (1 << 24)
     if uses_tensor:
         # Tensor contraction: one stream bit-op is one multiply-accumulate = 2 ops, run as 4-bit floating point
-        # (e2m1, tcgen05.mma kind::mxf4).  Peak for fp4 = the measured bf16 burst figure x the nominal ratio of the
-        # dense peaks (fp4 9 : bf16 2.25 PFLOP/s).
+        # (e2m1, tcgen05.mma kind::mxf4).  Two denominators: (a) the measured bf16 burst figure x the nominal ratio of the
+        # dense peaks (fp4 9 : bf16 2.25 PFLOP/s); (b) the issue rate of the core's own instruction, measured here by a
+        # bare chain of MMAs (multiply-accumulates per clock per SM) x SMs x the maximum SM clock.  `peak` is the larger.
         bf16 = peaks.get("bf16_tflops")
-        peak_tops = (bf16 if bf16 else 1590.0) * FP4_TO_BF16_NOMINAL
+        peak_a = (bf16 if bf16 else 1590.0) * FP4_TO_BF16_NOMINAL
+        mclk, macs = binding.sc_microbench(sc.ctx, 8, 4096)            # 128 x 192 x 64 block-scaled e2m1 MMAs
+        mac_per_clk_sm = macs / (mclk * 1e6)
+        peak_b = 2.0 * mac_per_clk_sm * n_sm * sm_max * 1e6 / 1e12
+        peak_tops = max(peak_a, peak_b)
+        ach = 2.0 * achieved / 1e12
         roofline = {
             "bound": "tensor",
             "kernel": "core_umma_kernel (tcgen05.mma kind::mxf4 on bits expanded on chip)",
-            "achieved": 2.0 * achieved / 1e12, "peak": peak_tops, "unit": "TFLOP/s", "frac": 2.0 * achieved / 1e12 / peak_tops,
+            "achieved": ach, "peak": peak_tops, "unit": "TFLOP/s", "frac": ach / peak_tops,
             "traffic": NCU_CORE_TRAFFIC_BYTES.get((w.name, "umma")),
-            "peak_source": ("measured bf16 burst %.1f TFLOP/s (MEASURED_PEAKS.json) x %g (nominal fp4 : bf16)"
-                            % (bf16, FP4_TO_BF16_NOMINAL))
-            if bf16 else "fallback 1590 TFLOP/s bf16 x %g (nominal fp4 : bf16)" % FP4_TO_BF16_NOMINAL,
+            "peak_source": ("the larger of (a) %s x %g (nominal fp4 : bf16) = %.0f TFLOP/s and (b) measured issue rate of "
+                            "the mxf4 MMA, %.0f MAC/clk/SM x %d SMs x %.0f MHz = %.0f TFLOP/s"
+                            % ("measured bf16 burst %.1f TFLOP/s (MEASURED_PEAKS.json)" % bf16 if bf16
+                               else "fallback 1590 TFLOP/s bf16", FP4_TO_BF16_NOMINAL, peak_a, mac_per_clk_sm, n_sm, sm_max,
+                               peak_b)),
+            "frac_vs_bf16_x4": ach / peak_a, "frac_vs_issue_rate": ach / peak_b,
+            "mxf4_mac_per_clk_per_sm": mac_per_clk_sm,
             "core_ms": core_avg_ms, "bitops_per_s": achieved, "times_popc_alu_bound": achieved / alu_peak,
             "hbm_gbs_measured_peak": peaks.get("hbm_gbs"),
         }
+        if clocks.get("sm_mhz"):
+            roofline["frac_vs_issue_rate_at_sampled_clock"] = ach / (peak_b * clocks["sm_mhz"] / sm_max)
     else:
         roofline = {
             "bound": "alu", "kernel": "core_kernel (gate + popcount accumulation)",
@@ -667,8 +703,9 @@ def main():
         for kind, name in ((0, "popc"), (4, "iadd3"), (2, "plain_mix_gates"), (3, "csa_mix_gates")):
             ms, words = binding.sc_microbench(sc.ctx, kind, 2000)
             mb[name + "_words_per_s"] = words / (ms * 1e-3)
-        mclk, macs = binding.sc_microbench(sc.ctx, 8 + 5, 4000)         # tcgen05 i8, A from tensor memory, N = 192
-        mb["tcgen05_i8_mac_per_clk_per_sm"] = macs / (mclk * 1e6)
+        for kind, name in ((8, "tcgen05_mxf4_n192_mac_per_clk_per_sm"), (9, "tcgen05_mxf4_n256_mac_per_clk_per_sm")):
+            mclk, macs = binding.sc_microbench(sc.ctx, kind, 4096)
+            mb[name] = macs / (mclk * 1e6)
         roofline["microbench"] = mb
 
     cpu_baseline = None
@@ -677,6 +714,27 @@ def main():
         dt = run()
         cpu_baseline = {"value": cb_bitops / dt, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
                         "seconds": dt}
+
+    # ---- the other benchmark configurations, a few steps each (recorded numbers beside the headline) -------
+    other = []
+    if not args.no_configs and world_size == 1:
+        del A, W, C, P, ws
+        torch.cuda.empty_cache()
+        for name in OTHER_CONFIGS:
+            m = measure_workload(sc, dev, name, args.core, reps=3)
+            core_rate = m["bitops"] / (m["core_ms"] * 1e-3)
+            entry = {"workload": name, "mode": m["mode"], "mean_L": round(m["mean_L"], 2), "step_ms": m["step_ms"],
+                     "core_ms": m["core_ms"], "prepared_step_ms": m["prepared_step_ms"],
+                     "step_bitops_per_s": m["bitops"] / (m["step_ms"] * 1e-3), "core_bitops_per_s": core_rate}
+            if m["tensor_core"] and roofline["bound"] == "tensor":
+                entry["core_frac"] = 2.0 * core_rate / 1e12 / roofline["peak"]
+                entry["core_frac_vs_bf16_x4"] = entry["core_frac"] / roofline["frac"] * roofline["frac_vs_bf16_x4"]
+            else:
+                entry["core_frac_alu"] = core_rate / alu_peak
+            other.append(entry)
+        status = sc.device_status()
+        if status != 0:
+            raise SystemExit("device status %d (%s) in the configs leg" % (status, binding.status_string(status)))
 
     mean_phase = {k: statistics.mean(p[k] for p in phases) for k in phases[0]}
     # achieved rates of the phases around the core (algorithmic bytes: fp32 operand read + packed planes written;
@@ -707,6 +765,7 @@ def main():
         "equiv_mac_per_s": float(w.M) * w.N * w.K * world_size * args.steps / (total_ms * 1e-3),
         "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
         "cpu_baseline": cpu_baseline, "phase_ms": mean_phase, "phase_rates": phase_rates,
+        "configs": other,
         "prepared_weights": {"value": bitops_per_step * world_size * args.steps / (prepared_ms * 1e-3), "unit": UNIT,
                              "ms_per_step": prepared_ms / args.steps,
                              "what": "same step through sc_matmul_prepared: the W-side encode is done once, outside "

@@ -60,6 +60,14 @@ enum { SC_CORE_AUTO = 0, SC_CORE_POPC = 1,   /* LOP3 + POPC on the integer pipes
        SC_CORE_SIMPLE = 3,                   /* one thread per output, no staging (debug reference)        */
        SC_CORE_UMMA = 4 };                   /* tcgen05 tensor cores (4-bit floats) on bits expanded on chip */
 
+/* Value -> comparator boundary (sc_params.quant).  Sec. 4.2 maps operands to the int8 grid (q_max = 127) and then to
+ * one of 257 comparison boundaries; how a grid point becomes a boundary is not printed. */
+enum { SC_QUANT_DIRECT257 = 0,       /* default: v = x / sigma straight onto the boundary grid, T = round((v + 1) 128)
+                                        (unipolar: round(|v| 256)): one rounding, E[decoded stream] = T / 128 - 1     */
+       SC_QUANT_INT8_THEN_257 = 1 }; /* the two steps of Sec. 4.2: x_hat = round(127 v) in -127..127, then the boundary
+                                        nearest to its stream probability (x_hat + 127) / 254 (Sec. 3.1) on the 0..256
+                                        scale, T = round((x_hat + 127) 128 / 127); unipolar: round(|x_hat| 256 / 127) */
+
 #define SC_L_CAP 1024           /* largest stream length accepted                                 */
 
 typedef struct {
@@ -70,6 +78,8 @@ typedef struct {
     uint64_t seed;        /* Philox key                                                          */
     uint32_t stream_id;   /* distinguishes calls that must not share streams (< 2^31)            */
     uint32_t core;        /* SC_CORE_*                                                           */
+    int32_t  quant;       /* SC_QUANT_*                                                          */
+    int32_t  reserved;    /* must be 0                                                           */
 } sc_params;
 
 /* ---- context ------------------------------------------------------------------------------- */
@@ -176,7 +186,7 @@ sc_status sc_matmul_batched(sc_ctx *ctx, const float *A, const float *W, int64_t
  * after W changes (the record cannot see that).
  *
  * sc_matmul_prepared is sc_matmul with the W-side work left out; results are identical bit for bit.
- * K and N come from the record.  params must repeat the mode, scale_w, seed and stream_id used at
+ * K and N come from the record.  params must repeat the mode, scale_w, quant, seed and stream_id used at
  * preparation (SC_ERR_ARG otherwise), Lmax may be anything up to the prepared one (SC_ERR_LENGTH beyond).
  * The buffer is laid out for the core chosen at preparation (params->core there, SC_CORE_AUTO rule on the
  * prepared Lmax): a later SC_CORE_AUTO follows it; an explicit core of the other family (tensor-core vs

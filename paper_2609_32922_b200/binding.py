@@ -18,6 +18,7 @@ SC_ERR_BUDGET, SC_ERR_WORKSPACE, SC_ERR_CUDA, SC_ERR_TIMEOUT = 5, 6, 7, 8
 SC_BIPOLAR_XNOR, SC_UNIPOLAR_AND = 0, 1
 SC_SCALE_NONE, SC_SCALE_PER_ROW, SC_SCALE_PER_TENSOR = 0, 1, 2
 SC_CORE_AUTO, SC_CORE_POPC, SC_CORE_CSA, SC_CORE_SIMPLE, SC_CORE_UMMA = 0, 1, 2, 3, 4
+SC_QUANT_DIRECT257, SC_QUANT_INT8_THEN_257 = 0, 1
 SC_L_CAP = 1024
 
 EXPORTS = (
@@ -33,7 +34,7 @@ EXPORTS = (
 class sc_params(ctypes.Structure):
     _fields_ = [("mode", ctypes.c_int32), ("scale_a", ctypes.c_int32), ("scale_w", ctypes.c_int32),
                 ("group", ctypes.c_int32), ("seed", ctypes.c_uint64), ("stream_id", ctypes.c_uint32),
-                ("core", ctypes.c_uint32)]
+                ("core", ctypes.c_uint32), ("quant", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 class ScError(RuntimeError):
@@ -121,8 +122,8 @@ def _check(code: int, where: str):
 
 
 def make_params(mode=SC_BIPOLAR_XNOR, scale_a=SC_SCALE_PER_ROW, scale_w=SC_SCALE_PER_TENSOR, group=1, seed=0,
-                stream_id=0, core=SC_CORE_AUTO) -> sc_params:
-    return sc_params(mode, scale_a, scale_w, group, seed, stream_id, core)
+                stream_id=0, core=SC_CORE_AUTO, quant=SC_QUANT_DIRECT257) -> sc_params:
+    return sc_params(mode, scale_a, scale_w, group, seed, stream_id, core, quant, 0)
 
 
 def _ptr(t) -> Optional[int]:

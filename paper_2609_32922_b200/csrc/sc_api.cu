@@ -83,6 +83,7 @@ static bool params_ok(const sc_params *p)
     if (p->group < 1) return false;
     if (p->stream_id >= (1u << 31)) return false;
     if (p->core > SC_CORE_UMMA) return false;
+    if ((p->quant != SC_QUANT_DIRECT257 && p->quant != SC_QUANT_INT8_THEN_257) || p->reserved != 0) return false;
     return true;
 }
 
@@ -267,6 +268,7 @@ sc_status sc_encode(sc_ctx *ctx, const float *X, int64_t rows, int64_t cols, int
     a.sigma = scales_out; a.seed = params->seed; a.stream_id = params->stream_id;
     a.streams = static_cast<uint32_t *>(streams_out); a.status = c->scratch + kSlotStatus;
     a.reverse_bytes = 0;
+    a.quant = params->quant;
     return launch_encode(a, st) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
 }
 
@@ -384,6 +386,7 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     ea.perm = perm; ea.l_sorted = l_sorted; ea.lmax_actual = c->scratch + kSlotLmaxActual; ea.Lmax = Lmax;
     ea.sigma = sigma_a; ea.seed = params->seed; ea.stream_id = params->stream_id;
     ea.streams = a_streams; ea.status = c->scratch + kSlotStatus; ea.reverse_bytes = 0;
+    ea.quant = params->quant;
     if (launch_encode(ea, st) != cudaSuccess) return SC_ERR_CUDA;
     mark(3);
     const bool and_form = umma && params->mode == SC_BIPOLAR_XNOR;    // AND counts + popcount corrections
@@ -519,11 +522,11 @@ sc_status sc_matmul_cbsg(sc_ctx *ctx, const float *A, const float *W, int64_t M,
     if (cudaMemsetAsync(acc, 0, sizeof(int32_t) * (size_t)M * (size_t)N, st) != cudaSuccess) return SC_ERR_CUDA;
     mark(2);
     if (launch_cbsg_encode(A, M, K, 0, w.m_pad, perm, l_sorted, c->scratch + kSlotLmaxActual, L, params->group, Lmax,
-                           sigma_a, tables, a_streams, 0, status, st) != cudaSuccess)
+                           sigma_a, tables, a_streams, 0, status, st, params->quant) != cudaSuccess)
         return SC_ERR_CUDA;
     mark(3);
     if (launch_cbsg_encode(W, K, N, 1, w.n_pad, nullptr, nullptr, c->scratch + kSlotLmaxActual, nullptr, 1, Lmax,
-                           sigma_w, tables, w_streams, 1, status, st) != cudaSuccess)
+                           sigma_w, tables, w_streams, 1, status, st, params->quant) != cudaSuccess)
         return SC_ERR_CUDA;
     mark(4);
     CoreArgs ca;
@@ -592,6 +595,7 @@ sc_status sc_weights_prepare(sc_ctx *ctx, const float *W, int64_t K, int64_t N, 
     ew.perm = nullptr; ew.l_sorted = nullptr; ew.lmax_actual = nullptr; ew.Lmax = Lmax;
     ew.sigma = sigma_w; ew.seed = params->seed; ew.stream_id = params->stream_id;
     ew.streams = w_streams; ew.status = c->scratch + kSlotStatus; ew.reverse_bytes = and_form ? 1 : (umma ? 2 : 0);
+    ew.quant = params->quant;
     if (launch_encode(ew, st) != cudaSuccess) return SC_ERR_CUDA;
     if (and_form && launch_col_corrections(w_streams, wl.n_pad, (int32_t)wl.kw, Lmax, nullptr, pop_w, st) != cudaSuccess)
         return SC_ERR_CUDA;
@@ -601,7 +605,7 @@ sc_status sc_weights_prepare(sc_ctx *ctx, const float *W, int64_t K, int64_t N, 
     h->magic = kWeightsMagic;
     h->device = c->device;
     h->K = K; h->N = N; h->Lmax = Lmax;
-    h->mode = params->mode; h->scale_w = params->scale_w;
+    h->mode = params->mode; h->scale_w = params->scale_w; h->quant = params->quant;
     h->seed = params->seed; h->stream_id = params->stream_id;
     h->umma = umma;
     h->sigma_w = sigma_w;
@@ -633,7 +637,7 @@ sc_status sc_matmul_prepared(sc_ctx *ctx, const float *A, const sc_weights *weig
     const sc_weights_impl *h = reinterpret_cast<const sc_weights_impl *>(weights);
     if (!ctx || !h || h->magic != kWeightsMagic || !params_ok(params)) return SC_ERR_ARG;
     if (h->device != reinterpret_cast<sc_ctx_impl *>(ctx)->device) return SC_ERR_ARG;
-    if (params->mode != h->mode || params->scale_w != h->scale_w || params->seed != h->seed ||
+    if (params->mode != h->mode || params->scale_w != h->scale_w || params->quant != h->quant || params->seed != h->seed ||
         params->stream_id != h->stream_id)
         return SC_ERR_ARG;
     if (Lmax > h->Lmax) return SC_ERR_LENGTH;

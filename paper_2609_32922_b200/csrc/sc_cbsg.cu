@@ -90,7 +90,7 @@ struct CbsgEncodeDev {
     const uint32_t *tables;
     uint32_t *streams;
     int32_t *status;
-    int32_t tensor_id, kw, group, Lmax, reverse_bytes;
+    int32_t tensor_id, kw, group, Lmax, reverse_bytes, quant;
 };
 
 __device__ __forceinline__ uint32_t low_bits(int32_t n)      // n lowest bits set, n clamped to 0..32
@@ -131,7 +131,8 @@ cbsg_encode_kernel(const __grid_constant__ CbsgEncodeDev p)
         if (src < 0 || !have_d) continue;
         float x = __ldg(p.X + (p.tensor_id == 0 ? src * p.x_cols + d : d * p.x_cols + src));
         if (is_nonfinite(x)) { bad = true; x = 0.0f; }
-        const int32_t T = boundary_bipolar(normalise(x, __ldg(p.sigma + src)));
+        const float v = normalise(x, __ldg(p.sigma + src));
+        const int32_t T = p.quant ? boundary_bipolar_int8(v) : boundary_bipolar(v);
         if (p.tensor_id == 0) {
             int32_t len = p.L ? __ldg(p.L + src / p.group) : p.Lmax;
             len = min(max(len, 0), p.Lmax);
@@ -244,7 +245,7 @@ cudaError_t launch_cbsg_encode(const float *X, int64_t rows, int64_t cols, int t
                                const int32_t *perm, const int32_t *l_sorted, const int32_t *lmax_actual,
                                const int32_t *L, int32_t group, int32_t Lmax, const float *sigma,
                                const uint32_t *tables, uint32_t *streams, int reverse_bytes, int32_t *status,
-                               cudaStream_t st)
+                               cudaStream_t st, int quant)
 {
     CbsgEncodeDev p;
     p.X = X; p.x_cols = cols;
@@ -254,6 +255,7 @@ cudaError_t launch_cbsg_encode(const float *X, int64_t rows, int64_t cols, int t
     p.perm = perm; p.l_sorted = l_sorted; p.lmax_actual = lmax_actual; p.L = L; p.sigma = sigma; p.tables = tables; p.streams = streams; p.status = status;
     p.tensor_id = tensor_id; p.kw = (int32_t)((p.depth + 31) / 32); p.group = group; p.Lmax = Lmax;
     p.reverse_bytes = reverse_bytes;
+    p.quant = quant;
     const int64_t warps = p.n_row_groups * p.kw;
     const int64_t blocks = (warps + 3) / 4;
     if (blocks <= 0) return cudaSuccess;

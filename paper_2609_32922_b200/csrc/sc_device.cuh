@@ -168,6 +168,23 @@ __device__ __forceinline__ int32_t boundary_unipolar(float v, uint32_t &negative
     return min(max(t, 0), 256);
 }
 
+// Two-step variant (Sec. 4.2): the int8 grid first (x_hat = round(127 v), binary32, round-half-even), then the nearest of
+// the 257 boundaries in integer arithmetic (127 is odd: no grid point lies half-way between two boundaries).
+__device__ __forceinline__ int32_t boundary_bipolar_int8(float v)
+{
+    int32_t q = __float2int_rn(__fmul_rn(v, 127.0f));
+    q = min(max(q, -127), 127);
+    return ((q + 127) * 256 + 127) / 254;
+}
+
+__device__ __forceinline__ int32_t boundary_unipolar_int8(float v, uint32_t &negative)
+{
+    negative = (v < 0.0f) ? 1u : 0u;
+    int32_t q = __float2int_rn(__fmul_rn(fabsf(v), 127.0f));
+    q = min(q, 127);
+    return (q * 512 + 127) / 254;
+}
+
 __device__ __forceinline__ bool is_nonfinite(float x)
 {
     return (__float_as_uint(x) & 0x7F800000u) == 0x7F800000u;

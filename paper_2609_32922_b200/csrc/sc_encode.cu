@@ -27,7 +27,7 @@ struct EncodeDev {
     const float *sigma;
     uint32_t *streams;
     int32_t *status;
-    int32_t tensor_id, kw, Lmax, n_chunks, chunk_blocks, reverse_bytes, vec_rows;
+    int32_t tensor_id, kw, Lmax, n_chunks, chunk_blocks, reverse_bytes, vec_rows, quant;
     uint32_t stream_word;
     // weight operand of a batched call: stream row r = b * batch_pad + j is output column j of product b, stored at
     // X[b][d][j] (or X[b][j][d] when transposed); batch_pad = 0 otherwise
@@ -135,8 +135,8 @@ encode_kernel(const __grid_constant__ PhiloxKeys ks, const __grid_constant__ Enc
             float xv = x[t];
             if (is_nonfinite(xv)) { bad = true; xv = 0.0f; }
             const float v = normalise(xv, sg[t]);
-            if (kMode == SC_BIPOLAR_XNOR) T = boundary_bipolar(v);
-            else T = boundary_unipolar(v, neg);
+            if (kMode == SC_BIPOLAR_XNOR) T = p.quant ? boundary_bipolar_int8(v) : boundary_bipolar(v);
+            else T = p.quant ? boundary_unipolar_int8(v, neg) : boundary_unipolar(v, neg);
             elem[t] = (uint64_t)(base[t] + d * d_stride);
         }
         info[t] |= T;
@@ -206,6 +206,7 @@ cudaError_t launch_encode(const EncodeArgs &a, cudaStream_t st)
     p.perm = a.perm; p.l_sorted = a.l_sorted; p.lmax_actual = a.lmax_actual; p.sigma = a.sigma;
     p.streams = a.streams; p.status = a.status;
     p.tensor_id = a.tensor_id; p.kw = (int32_t)a.kw; p.Lmax = a.Lmax; p.reverse_bytes = a.reverse_bytes;
+    p.quant = a.quant;
     p.stream_word = ((uint32_t)a.tensor_id & 1u) | (a.stream_id << 1);
     p.batch_pad = a.batch_pad; p.batch_real = a.batch_real; p.w_transposed = a.w_transposed;
     // W read as two 16-byte vectors per lane when its rows keep them aligned

@@ -94,7 +94,7 @@ struct sc_weights_impl {
     int device;
     int64_t K, N;
     int32_t Lmax;
-    int mode, scale_w;
+    int mode, scale_w, quant;
     uint64_t seed;
     uint32_t stream_id;
     bool umma;               // laid out for the tensor-core core (else for the ALU cores)
@@ -150,6 +150,7 @@ struct EncodeArgs {
     int64_t batch_pad = 0;       // padded stream rows per product (0: not batched, rows = stream rows)
     int64_t batch_real = 0;      // real stream rows per product
     int w_transposed = 0;        // X stored [B][N][K] instead of [B][K][N]
+    int quant = 0;               // SC_QUANT_*: value -> boundary rule
 };
 cudaError_t launch_encode(const EncodeArgs &a, cudaStream_t st);
 cudaError_t launch_unpack(const uint32_t *streams, int64_t stream_rows, int64_t depth, int32_t Lmax, int mode,
@@ -197,7 +198,7 @@ cudaError_t launch_cbsg_encode(const float *X, int64_t rows, int64_t cols, int t
                                const int32_t *perm, const int32_t *l_sorted, const int32_t *lmax_actual,
                                const int32_t *L, int32_t group, int32_t Lmax, const float *sigma,
                                const uint32_t *tables, uint32_t *streams, int reverse_bytes, int32_t *status,
-                               cudaStream_t st);
+                               cudaStream_t st, int quant = 0);
 cudaError_t launch_cbsg_scc(const uint32_t *tables, const int32_t *Ta, const int32_t *Tw, int64_t n, int32_t L,
                             int32_t *counts, double *scc, int32_t *status, cudaStream_t st);
 cudaError_t launch_cbsg_decode(const int32_t *acc, int64_t M, int64_t N, int64_t K, const int32_t *L, int32_t group,

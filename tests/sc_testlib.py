@@ -33,9 +33,9 @@ def gpu_matmul(sc, binding, w, A, W, L_groups, Lmax, group=1, core=0, want_P=Tru
     return (None if P is None else P.cpu().numpy()), C.cpu().numpy()
 
 
-def oracle_matmul(oracle, w, A, W, L_rows, rows=None, cols=None):
+def oracle_matmul(oracle, w, A, W, L_rows, rows=None, cols=None, quant=0):
     return oracle.matmul(A, W, L_rows, MODES[w.mode], SCALES[w.scale_a], SCALES[w.scale_w], w.seed, w.stream_id,
-                         row_sel=rows, col_sel=cols)
+                         row_sel=rows, col_sel=cols, quant=quant)
 
 
 def policy_lengths(oracle, w, A):

@@ -32,7 +32,7 @@ def test_reference_arm_json_line():
 
 @pytest.mark.gpu
 def test_cuda_arm_json_line():
-    d = _run("--steps", "3", "--warmup", "3", "--no-cpu-baseline")
+    d = _run("--steps", "3", "--warmup", "3", "--no-cpu-baseline", "--no-configs")
     for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
                 "vs_baseline", "dtype", "data", "config", "e2e", "gpu_launches", "clocks", "roofline"):
         assert key in d, key
@@ -40,4 +40,7 @@ def test_cuda_arm_json_line():
     assert d["e2e"]["h2d_bytes_per_step"] > 0 and d["e2e"]["d2h_bytes_per_step"] > 0 and 0 < d["e2e"]["value"] <= d["value"] * 1.05
     r = d["roofline"]
     assert r["bound"] == "tensor" and 0.3 < r["frac"] < 1.1 and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
+    # both denominators are reported; `peak` is the larger one, so `frac` is the smaller fraction
+    assert r["frac"] <= min(r["frac_vs_bf16_x4"], r["frac_vs_issue_rate"]) + 1e-12
+    assert 8000 < r["mxf4_mac_per_clk_per_sm"] < 17000
     assert d["clocks"]["sm_max_mhz"] >= d["clocks"]["sm_mhz"] > 0

@@ -26,9 +26,10 @@ def sc(binding):
     s.close()
 
 
-def _run(sc, binding, A, W, L, Lmax, scale_a, scale_w, seed, stream_id=0, group=1, want_P=True):
+def _run(sc, binding, A, W, L, Lmax, scale_a, scale_w, seed, stream_id=0, group=1, want_P=True, quant=0):
     import torch
-    params = binding.make_params(mode=0, scale_a=scale_a, scale_w=scale_w, group=group, seed=seed, stream_id=stream_id)
+    params = binding.make_params(mode=0, scale_a=scale_a, scale_w=scale_w, group=group, seed=seed, stream_id=stream_id,
+                                 quant=quant)
     dL = None if L is None else torch.from_numpy(np.ascontiguousarray(L, dtype=np.int32)).cuda()
     P, C = sc.matmul_cbsg(torch.from_numpy(A).cuda(), torch.from_numpy(W).cuda(), dL, Lmax, params, want_P)
     torch.cuda.synchronize()
@@ -49,6 +50,21 @@ def test_small_ragged_full(sc, binding, oracle, seed, scale_w):
     assert np.array_equal(P, ref["P"])
     assert T.close_enough(C, ref["C"])
     assert (C[0] == 0).all()
+
+
+def test_int8_grid_first_as_in_the_papers_datapath(sc, binding, oracle):
+    """The fused quantisation of Sec. 4.2 in two steps (int8 grid, then one of the 257 boundaries): counts equal the oracle's
+    with the same rule and differ from the direct rule's."""
+    rng = np.random.default_rng(12)
+    M, K, N = 150, 96, 200
+    A = rng.standard_normal((M, K)).astype(np.float32)
+    W = (0.02 * rng.standard_normal((K, N))).astype(np.float32)
+    L = rng.integers(0, 257, size=M).astype(np.int32)
+    P, C = _run(sc, binding, A, W, L, 256, PER_ROW, PER_TENSOR, 6, stream_id=1, quant=binding.SC_QUANT_INT8_THEN_257)
+    ref = oracle.matmul_cbsg(A, W, L, PER_ROW, PER_TENSOR, seed=6, stream_id=1, quant=oracle.QUANT_INT8_THEN_257)
+    assert np.array_equal(P, ref["P"]) and T.close_enough(C, ref["C"])
+    direct = oracle.matmul_cbsg(A, W, L, PER_ROW, PER_TENSOR, seed=6, stream_id=1)
+    assert not np.array_equal(P, direct["P"])
 
 
 def test_groups_uniform_and_exact_full_length(sc, binding, oracle):

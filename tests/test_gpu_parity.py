@@ -96,6 +96,33 @@ def test_small_ragged_full(sc, binding, oracle, mode, core):
     assert (C[0] == 0).all() and (P[0] == 0).all()
 
 
+@pytest.mark.parametrize("mode", ["bipolar", "unipolar"])
+def test_int8_grid_first_quantisation(sc, binding, oracle, mode):
+    """sc_params.quant = SC_QUANT_INT8_THEN_257: boundaries through the int8 grid (Sec. 4.2), streams and counts equal
+    the oracle's with the same rule; prepared weights carry the rule."""
+    import torch
+    w, L_rows = wl.small_ragged(seed=17, mode=mode)
+    A, W = wl.make_inputs(w)
+    params = T.gpu_params(binding, w)
+    params.quant = binding.SC_QUANT_INT8_THEN_257
+    dA, dW, dL = torch.from_numpy(A).cuda(), torch.from_numpy(W).cuda(), torch.from_numpy(L_rows).cuda()
+    P, C = sc.matmul(dA, dW, dL, 100, params)
+    torch.cuda.synchronize()
+    ref = T.oracle_matmul(oracle, w, A, W, L_rows, quant=oracle.QUANT_INT8_THEN_257)
+    assert np.array_equal(P.cpu().numpy(), ref["P"]) and T.close_enough(C.cpu().numpy(), ref["C"])
+    assert not np.array_equal(ref["P"], T.oracle_matmul(oracle, w, A, W, L_rows)["P"])
+    prepared = sc.prepare_weights(dW, 100, params)
+    ws = sc.workspace(binding.sc_workspace_bytes_prepared(w.M, w.K, w.N, 100, params))
+    P2, C2 = torch.empty_like(P), torch.empty_like(C)
+    binding.sc_matmul_prepared(sc.ctx, dA, prepared[0], dL, 100, params, P2, C2, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(P, P2) and torch.equal(C, C2)
+    other = T.gpu_params(binding, w)                                 # the direct rule: the record refuses it
+    with pytest.raises(binding.ScError):
+        binding.sc_matmul_prepared(sc.ctx, dA, prepared[0], dL, 100, other, P2, C2, ws)
+    binding.sc_weights_release(prepared[0])
+
+
 def test_groups_and_accumulator_workspace(sc, binding, oracle):
     """Lengths per group of 8 rows (last group short); P not requested (accumulators live in the workspace)."""
     w, _ = wl.small_ragged(seed=5, M=150, K=96, N=130)
