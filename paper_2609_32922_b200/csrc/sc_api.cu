@@ -27,7 +27,10 @@ Workspace layout_workspace(int64_t M, int64_t K, int64_t N, int32_t Lmax, int mo
     M *= B;
     N *= B;
     w.kw = (K + 31) / 32;
-    w.a_planes = (int64_t)Lmax * w.kw * ppq;
+    // unipolar: the tensor-core core stores the positions in blocks (lengths rounded up to whole blocks); the planes are
+    // sized so that either core family fits (two planes per position; the tensor-core core's W uses one of them)
+    const int64_t l_alloc = mode == SC_UNIPOLAR_AND ? round_up(Lmax, kPosBlockSigned) : Lmax;
+    w.a_planes = l_alloc * w.kw * ppq;
     w.w_planes = w.a_planes;
     const int64_t n_row_tiles = w.m_pad / kTileM;
     size_t off = 0;
@@ -43,6 +46,8 @@ Workspace layout_workspace(int64_t M, int64_t K, int64_t N, int32_t Lmax, int mo
     w.pop_w = take(with_w ? sizeof(int32_t) * (size_t)(Lmax + 1) * (size_t)w.n_pad : 0);
     w.a_streams = take(sizeof(uint32_t) * (size_t)w.a_planes * (size_t)w.m_pad);
     w.w_streams = take(with_w ? sizeof(uint32_t) * (size_t)w.w_planes * (size_t)w.n_pad : 0);
+    w.w_sign = take(with_w && mode == SC_UNIPOLAR_AND ? 4 * sizeof(uint32_t) * (size_t)w.kw * (size_t)w.n_pad : 0);
+    w.a_sign = take(mode == SC_UNIPOLAR_AND ? 4 * sizeof(uint32_t) * (size_t)w.kw * (size_t)w.m_pad : 0);
     w.total = off;
     return w;
 }
@@ -53,12 +58,14 @@ WeightsLayout layout_weights(int64_t K, int64_t N, int32_t Lmax, int mode)
     memset(&w, 0, sizeof(w));
     w.n_pad = round_up(N, kColPad);
     w.kw = (K + 31) / 32;
-    w.w_planes = (int64_t)Lmax * w.kw * planes_per_step(mode);
+    const int64_t l_alloc = mode == SC_UNIPOLAR_AND ? round_up(Lmax, kPosBlockSigned) : Lmax;
+    w.w_planes = l_alloc * w.kw * planes_per_step(mode);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes, 256); return at; };
     w.sigma_w = take(sizeof(float) * (size_t)N);
     w.pop_w = take(sizeof(int32_t) * (size_t)(Lmax + 1) * (size_t)w.n_pad);
     w.w_streams = take(sizeof(uint32_t) * (size_t)w.w_planes * (size_t)w.n_pad);
+    w.w_sign = take(mode == SC_UNIPOLAR_AND ? 4 * sizeof(uint32_t) * (size_t)w.kw * (size_t)w.n_pad : 0);
     w.total = off;
     return w;
 }
@@ -339,7 +346,13 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     const uint32_t *w_streams = pw ? pw->w_streams : w_streams_ws;
     int32_t *pop_w_ws = reinterpret_cast<int32_t *>(base + w.pop_w);
     const int32_t *pop_w = pw ? pw->pop_w : pop_w_ws;
-    const int ppq = planes_per_step(params->mode);
+    const int ppq_alloc = planes_per_step(params->mode);                 // planes per position the buffers are sized for
+    const int ppq = planes_per_step_for(params->mode, umma);             // ... and as written for the core that runs
+    const int pos_block = pos_block_for(params->mode, umma);
+    uint32_t *w_sign_ws = reinterpret_cast<uint32_t *>(base + w.w_sign);
+    const uint32_t *w_sign = pw ? pw->w_sign : w_sign_ws;
+    uint32_t *a_sign = reinterpret_cast<uint32_t *>(base + w.a_sign);
+    const bool signs = umma && params->mode == SC_UNIPOLAR_AND;
 
     auto mark = [&](int k) { if (c->profiling) cudaEventRecord(c->phase_ev[k], st); };
     c->profile_valid = false;
@@ -361,7 +374,7 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     // a3: row ordering by length and the work list
     auto plan_rows = [&]() -> bool {
         if (launch_plan(L, M, params->group, Lmax, w.kw, ppq, m_pad_b, n_col_tiles, umma ? 0 : c->sm_count * 16,
-                        umma ? c->sm_count : 0, l_rows, perm, l_sorted, plan, c->scratch, st, B) != cudaSuccess)
+                        umma ? c->sm_count : 0, l_rows, perm, l_sorted, plan, c->scratch, st, B, pos_block) != cudaSuccess)
             return false;
         // the W encode stops at the longest length of the call
         if (fork && (cudaEventRecord(c->ev_plan, st) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_plan, 0) != cudaSuccess))
@@ -387,6 +400,8 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     ea.sigma = sigma_a; ea.seed = params->seed; ea.stream_id = params->stream_id;
     ea.streams = a_streams; ea.status = c->scratch + kSlotStatus; ea.reverse_bytes = 0;
     ea.quant = params->quant;
+    ea.pos_block = pos_block;
+    ea.signs = signs ? a_sign : nullptr;
     if (launch_encode(ea, st) != cudaSuccess) return SC_ERR_CUDA;
     mark(3);
     const bool and_form = umma && params->mode == SC_BIPOLAR_XNOR;    // AND counts + popcount corrections
@@ -397,7 +412,8 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
         ew.w_transposed = w_transposed;
         if (B > 1) { ew.batch_pad = n_pad_b; ew.batch_real = N; }
         ew.perm = nullptr; ew.l_sorted = nullptr; ew.sigma = sigma_w_ws; ew.streams = w_streams_ws;
-        ew.reverse_bytes = and_form ? 1 : (umma ? 2 : 0);
+        ew.reverse_bytes = umma ? 1 : 0;
+        ew.signs = signs ? w_sign_ws : nullptr;
         if (launch_encode(ew, sw) != cudaSuccess) return SC_ERR_CUDA;
         if (and_form && launch_col_corrections(w_streams_ws, w.n_pad, (int32_t)w.kw, Lmax,
                                                c->scratch + kSlotLmaxActual, pop_w_ws, sw) != cudaSuccess)
@@ -409,7 +425,10 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     // a5-a7: gate + popcount accumulation
     CoreArgs ca;
     ca.a_streams = a_streams; ca.w_streams = w_streams;
-    ca.m_pad = w.m_pad; ca.n_pad = w.n_pad; ca.a_planes = w.a_planes; ca.w_planes = w.w_planes;
+    ca.m_pad = w.m_pad; ca.n_pad = w.n_pad;
+    ca.a_planes = w.a_planes / ppq_alloc * ppq;                          // planes the operands really have
+    ca.w_planes = w.w_planes / ppq_alloc * ppq;
+    ca.w_sign = signs ? w_sign : nullptr; ca.a_sign = signs ? a_sign : nullptr; ca.pos_block = pos_block;
     ca.M = Mt; ca.N = N; ca.mode = params->mode;
     ca.tiles_m = (int32_t)(m_pad_b / kTileM); ca.w_batch_cols = n_pad_b;
     ca.variant = variant;
@@ -594,8 +613,12 @@ sc_status sc_weights_prepare(sc_ctx *ctx, const float *W, int64_t K, int64_t N, 
     ew.stream_rows = N; ew.depth = K; ew.kw = wl.kw; ew.r_pad = wl.n_pad;
     ew.perm = nullptr; ew.l_sorted = nullptr; ew.lmax_actual = nullptr; ew.Lmax = Lmax;
     ew.sigma = sigma_w; ew.seed = params->seed; ew.stream_id = params->stream_id;
-    ew.streams = w_streams; ew.status = c->scratch + kSlotStatus; ew.reverse_bytes = and_form ? 1 : (umma ? 2 : 0);
+    ew.streams = w_streams; ew.status = c->scratch + kSlotStatus; ew.reverse_bytes = umma ? 1 : 0;
     ew.quant = params->quant;
+    ew.pos_block = pos_block_for(params->mode, umma);
+    uint32_t *w_sign = reinterpret_cast<uint32_t *>(base + wl.w_sign);
+    const bool signs = umma && params->mode == SC_UNIPOLAR_AND;
+    ew.signs = signs ? w_sign : nullptr;
     if (launch_encode(ew, st) != cudaSuccess) return SC_ERR_CUDA;
     if (and_form && launch_col_corrections(w_streams, wl.n_pad, (int32_t)wl.kw, Lmax, nullptr, pop_w, st) != cudaSuccess)
         return SC_ERR_CUDA;
@@ -611,6 +634,7 @@ sc_status sc_weights_prepare(sc_ctx *ctx, const float *W, int64_t K, int64_t N, 
     h->sigma_w = sigma_w;
     h->pop_w = and_form ? pop_w : nullptr;
     h->w_streams = w_streams;
+    h->w_sign = signs ? w_sign : nullptr;
     *out = reinterpret_cast<sc_weights *>(h);
     return SC_OK;
 }
@@ -736,19 +760,32 @@ int32_t sc_selftest_expansion(void)
         u_expand_bits<false>(za, ea);
         u_expand_bits<true>(w_plane, ew);
         if (expanded_dot(ea, ew) != (double)__builtin_popcount(za & zw)) ++mismatches;
-        // unipolar: magnitude / negative planes against the two field planes; signs count only where the stream bit is set
-        const uint32_t na = za & sa, nw = zw & sw;
-        uint32_t p0, p1;
-        pack_w_fields(zw, nw, p0, p1);
-        u_expand_signed_w(p0, p1, ew);
+        // unipolar: magnitude planes (the weight's in reversed order) with the nibble sign words of the elements' signs;
+        // signs count only where both stream bits are set
+        uint32_t w_sign = 0u;
+        for (int b = 0; b < 32; ++b) w_sign |= ((sw >> w_bit_element(b)) & 1u) << b;
+        uint32_t sn_a[4], sn_w[4];
+        sign_nibble_words(sa, false, sn_a);
+        sign_nibble_words(w_sign, true, sn_w);
+        u_expand_signed<false>(za, sn_a, ea);
+        u_expand_signed<true>(w_plane, sn_w, ew);
         int32_t expect = 0;
         for (int e = 0; e < 32; ++e)
-            if ((za >> e) & (zw >> e) & 1u) expect += (((na >> e) ^ (nw >> e)) & 1u) ? -1 : 1;
-        u_expand_signed_a(za, na, ea, true);
+            if ((za >> e) & (zw >> e) & 1u) expect += (((sa >> e) ^ (sw >> e)) & 1u) ? -1 : 1;
         if (expanded_dot(ea, ew) != (double)expect) ++mismatches;
-        if (na == 0u) {                    // the unsigned rule for activations without a negative stream bit
-            u_expand_signed_a(za, 0u, ea, false);
+        if ((za & sa) == 0u) {             // the unsigned rule for activations without a negative stream bit
+            u_expand_bits<false>(za, ea);
             if (expanded_dot(ea, ew) != (double)expect) ++mismatches;
+        }
+        // position blocks: every (position, depth word) pair of a stream of 21 positions x 5 depth words gets its own plane
+        if (trial == 0) {
+            bool seen[24 * 5] = {false};
+            for (int l = 0; l < 21; ++l)
+                for (int w = 0; w < 5; ++w) {
+                    const int64_t pi = plane_index(l, w, 5, kPosBlockSigned);
+                    if (pi < 0 || pi >= 24 * 5 || seen[pi]) ++mismatches; else seen[pi] = true;
+                    if (plane_index(l, w, 5, 1) != (int64_t)l * 5 + w) ++mismatches;
+                }
         }
     }
     return mismatches;

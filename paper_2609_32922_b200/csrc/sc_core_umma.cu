@@ -13,8 +13,10 @@
 //   bipolar : a set bit becomes a power of two chosen so that every product is exactly 1; the MMA yields the AND
 //             count, and the decode pass turns it into the XNOR count,
 //             XNOR = K L_i - pop(A_i, l < L_i) - pop(W_j, l < L_i) + 2 AND;
-//   unipolar: signed nibbles, +-0.5 (magnitude and negative planes) against +-2 (two-bit fields); the MMA yields the
-//             signed count directly.
+//   unipolar: the same powers of two with a sign bit: both operands come as magnitude planes plus, per (depth word,
+//             row / column), the signs of its 32 elements as four nibble words (the activations' are skipped when the
+//             call has no negative stream bit); positions are stored in blocks of 8 so that an operand stage is 8
+//             positions of one depth word and one set of sign words serves the stage; the MMA yields the signed count.
 //
 // Warp roles (one CTA of 28 warps per SM, persistent; each CTA owns an equal contiguous run of the stage units of all
 // tiles, see u_piece):
@@ -32,6 +34,8 @@
 // factors.
 // Every wait is bounded; a wait that runs out sets SC_ERR_TIMEOUT and records where, all roles drain, tensor
 // memory is freed.
+#include <type_traits>
+
 #include "sc_device.cuh"
 #include "sc_internal.h"
 
@@ -103,9 +107,13 @@ struct UmmaDev {
     int32_t *acc;
     int32_t *scratch;
     int64_t N;
-    int32_t planes_per_len;
+    int32_t planes_per_len;           // W planes (= K-step halves) per stream position: the depth words
+    int32_t pos_block;                // stream positions are stored in blocks of this many (1: position-major)
     int32_t tiles_m;                  // row tiles per product (batched calls stack products along rows / columns)
     int64_t w_batch_cols;             // padded W stream rows per product
+    const uint32_t *w_sign;           // unipolar: [depth word][n_pad][4] nibble sign words of W ...
+    const uint32_t *a_sign;           // ... and [depth word][m_pad][4] of A
+    int64_t n_pad;                    // padded W stream rows in all
 };
 
 __device__ __forceinline__ uint32_t u_smem(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -255,11 +263,12 @@ template <int kMode>
 __global__ void __launch_bounds__(kUThreads, 1)
 core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
 {
-    // raw planes per MMA K-step of 64 elements: two (depth word, position) pairs, each one plane (bipolar) or two
-    // (unipolar: magnitude + negative, or the weight's two field planes)
-    constexpr int kPpq = kMode == SC_UNIPOLAR_AND ? 4 : 2;
+    // An MMA K-step of 64 elements is two (depth word, position) pairs = two planes of either operand.
+    constexpr int kPpq = 2;
     constexpr int kStepsPerRaw = kStagePlanes / kPpq;              // MMA steps in one raw stage
     constexpr int kOpsPerRaw = kStepsPerRaw / kOpSteps;            // operand stages in one raw stage
+    constexpr int kStagePp = kOpSteps * kPpq;                      // (depth word, position) pairs of one operand stage
+    static_assert(kStagePp == kPosBlockSigned, "a signed operand stage is one block of positions of one depth word");
 
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t *raw = smem;
@@ -438,7 +447,8 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
             pos += it.n_raw;
             const int64_t r = (int64_t)it.rt * kTileM + quarter * 32 + lane;
             int32_t src = __ldg(p.perm + r);
-            if (__ldg(p.l_sorted + r) * p.planes_per_len <= it.q0) src = -1;       // nothing of this row in the chunk
+            // nothing of this row in the chunk: its stream ends at or before the first position block of the chunk
+            if (__ldg(p.l_sorted + r) <= it.q0 / (p.pos_block * p.planes_per_len) * p.pos_block) src = -1;
             const uint32_t b = single ? 0u : acc_cnt & 1u, acc_phase = (single ? acc_cnt : acc_cnt >> 1) & 1u;
             if (!u_mbar_wait_warp(bar(kAccFull + b), acc_phase, s_abort, lane)) { if (lane == 0) give_up(5, acc_cnt, 0); break; }
             u_fence_after();
@@ -492,10 +502,16 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
         const uint32_t quarter = (uint32_t)warp & 3u;
         const int group = (warp - kAFirstWarp) / kAWarps;
         const int row = (int)(quarter * 32 + lane);
-        const bool a_signed = kMode == SC_UNIPOLAR_AND && __ldg(p.scratch + kSlotAnyNegA) != 0;
-        constexpr int kStagePl = kOpSteps * kPpq;     // raw planes of one operand stage
+        // Unipolar activations without a negative stream bit in the call (post-ReLU / GELU outputs, attention
+        // probabilities) skip the sign words; the two cases are compiled separately so that the unsigned one carries no
+        // registers for them.
+        const bool a_signed_call = kMode == SC_UNIPOLAR_AND && __ldg(p.scratch + kSlotAnyNegA) != 0;
+        auto run_expander = [&](auto signed_tag) {
+        constexpr bool a_signed = decltype(signed_tag)::value;
+        constexpr int kStagePl = kStagePp;            // A plane words of one operand stage held in registers
+        constexpr int kSignWords = a_signed ? 4 : 1;
         struct AIter {
-            int32_t pos, end, j, n_ops, my_end, rt, q0, n_raw;
+            int32_t pos, end, j, n_ops, my_len, rt, q0, q1, n_raw;
             uint32_t op;
             bool valid;
         };
@@ -503,11 +519,10 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
             x.valid = x.pos < x.end;
             if (!x.valid) return;
             const UItem it = u_piece(plan, prefix, tile_planes, x.pos, x.end);
-            x.rt = it.rt; x.q0 = it.q0; x.n_raw = it.n_raw;
+            x.rt = it.rt; x.q0 = it.q0; x.q1 = it.q1; x.n_raw = it.n_raw;
             x.n_ops = it.n_raw * kOpsPerRaw;
             x.j = 0;
-            // a row contributes planes below min(its own end, the end of this piece)
-            x.my_end = min(__ldg(p.l_sorted + (int64_t)it.rt * kTileM + row) * p.planes_per_len, it.q1);
+            x.my_len = __ldg(p.l_sorted + (int64_t)it.rt * kTileM + row);
         };
         auto advance = [&](AIter &x, int n) {
             for (int a = 0; a < n && x.valid; ++a) {
@@ -515,15 +530,21 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
                 if (++x.j == x.n_ops) { x.pos += x.n_raw; load_piece(x); }
             }
         };
-        auto fetch = [&](const AIter &x, uint32_t (&dst)[kStagePl]) {
-            const int32_t q_abs = x.q0 + x.j * kStagePl;
-            const uint32_t *src = p.a_streams + (int64_t)q_abs * p.m_pad + (int64_t)x.rt * kTileM + row;
+        auto fetch = [&](const AIter &x, uint32_t (&dst)[kStagePl], uint32_t (&sgn)[kSignWords]) {
+            const int32_t pp0 = x.q0 + x.j * kStagePp;              // first (depth word, position) pair of the stage
+            // A row contributes the pairs below the end of this piece whose position lies below its own length; in a
+            // stage these are the leading ones: position-major, the pairs below l_i * (depth words); in blocks of 8
+            // positions, the stage is positions lb .. lb + 7 of one depth word.
+            int32_t n_act;
+            if (p.pos_block == 1) n_act = min(x.my_len * p.planes_per_len, x.q1) - pp0;
+            else n_act = min(x.my_len - pp0 / (kPosBlockSigned * p.planes_per_len) * kPosBlockSigned, x.q1 - pp0);
+            const uint32_t *src = p.a_streams + (int64_t)pp0 * p.m_pad + (int64_t)x.rt * kTileM + row;
 #pragma unroll
-            for (int q = 0; q < kStagePl; ++q) {
-                // planes at or beyond the row's end are zero; unipolar activations without a negative stream bit do
-                // not read the negative planes
-                const bool skip = kMode == SC_UNIPOLAR_AND && !a_signed && (q & 1);
-                dst[q] = (!skip && q_abs + q < x.my_end) ? __ldcs(src + (int64_t)q * p.m_pad) : 0u;
+            for (int q = 0; q < kStagePl; ++q) dst[q] = q < n_act ? __ldcs(src + (int64_t)q * p.m_pad) : 0u;
+            if (a_signed) {
+                const int32_t wd = pp0 % (kPosBlockSigned * p.planes_per_len) / kPosBlockSigned;
+                const uint4 v = __ldg(reinterpret_cast<const uint4 *>(p.a_sign) + (int64_t)wd * p.m_pad + (int64_t)x.rt * kTileM + row);
+                sgn[0] = v.x; sgn[1 % kSignWords] = v.y; sgn[2 % kSignWords] = v.z; sgn[3 % kSignWords] = v.w;
             }
         };
         AIter cur;
@@ -532,11 +553,11 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
         advance(cur, group);
         AIter nxt = cur;
         advance(nxt, kAGroups);
-        uint32_t now[kStagePl], ahead[kStagePl];
-        if (cur.valid) fetch(cur, now);
+        uint32_t now[kStagePl], ahead[kStagePl], now_s[kSignWords], ahead_s[kSignWords];
+        if (cur.valid) fetch(cur, now, now_s);
         bool ok = true;
         while (cur.valid && ok && !*s_abort) {
-            if (nxt.valid) fetch(nxt, ahead);
+            if (nxt.valid) fetch(nxt, ahead, ahead_s);
             const uint32_t op_cnt = cur.op, t = op_cnt % kOpStages;
             // The slot of the A ring (depth D) was last read by the MMAs of operand stage op_cnt - D; its barrier is the
             // "stage free" barrier of that operand stage (even and odd uses of a W stage signal different barriers).
@@ -559,12 +580,12 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
 #pragma unroll
             for (int st = 0; st < kOpSteps; ++st) {
                 uint32_t out[8];
-                if (kMode == SC_BIPOLAR_XNOR) {
+                if (!a_signed) {
                     u_expand_bits<false>(now[2 * st], out);
                     u_expand_bits<false>(now[2 * st + 1], out + 4);
                 } else {
-                    u_expand_signed_a(now[4 * st], now[4 * st + 1], out, a_signed);
-                    u_expand_signed_a(now[4 * st + 2], now[4 * st + 3], out + 4, a_signed);
+                    u_expand_signed<false>(now[2 * st], now_s, out);
+                    u_expand_signed<false>(now[2 * st + 1], now_s, out + 4);
                 }
                 u_tmem_st8(a_col + st * 8u, out);
             }
@@ -574,10 +595,19 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
             if (lane == 0) u_mbar_arrive(bar(kOpFull + t));
 #pragma unroll
             for (int q = 0; q < kStagePl; ++q) now[q] = ahead[q];
+#pragma unroll
+            for (int q = 0; q < kSignWords; ++q) now_s[q] = ahead_s[q];
             cur = nxt;
             advance(nxt, kAGroups);
         }
         if (!ok && lane == 0) give_up(7, cur.op, 0);
+        };
+        if constexpr (kMode == SC_UNIPOLAR_AND) {
+            if (a_signed_call) run_expander(std::true_type{});
+            else run_expander(std::false_type{});
+        } else {
+            run_expander(std::false_type{});
+        }
     } else {
         // ---------------- W expanders: two columns per thread, bit planes from the TMA ring into shared memory ----
         const int group = (warp - kWFirstWarp) / kWWarps;
@@ -590,25 +620,48 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
             pos += it.n_raw;
             for (int32_t k = 0; k < (it.n_raw + kRawUnits - 1) / kRawUnits && ok; ++k, ++raw_cnt) {
                 const uint32_t s = raw_cnt % kRawStages;
+                const int ops_here = min(kRawUnits, it.n_raw - k * kRawUnits) * kOpsPerRaw;    // units present in this box
+                // Unipolar: the sign words of this group's stages of the box (a box holds kRawUnits * kOpsPerRaw stages, the
+                // group fills every kWGroups-th) are requested from global memory before the box is awaited, so that their
+                // latency hides behind that wait.  A stage is eight positions of one depth word: one sign word per column.
+                constexpr int kOwnMax = (kRawUnits * kOpsPerRaw + kWGroups - 1) / kWGroups;
+                uint4 sg_box[kOwnMax][kWCols];
+                if (kMode == SC_UNIPOLAR_AND) {
+                    const int first_own = (group + kWGroups - (int)(op_cnt % kWGroups)) % kWGroups;
+                    const uint4 *sign_col = reinterpret_cast<const uint4 *>(p.w_sign) + (int64_t)(it.rt / p.tiles_m) * p.w_batch_cols +
+                                            (int64_t)it.ct * kUN + row;
+#pragma unroll
+                    for (int o = 0; o < kOwnMax; ++o) {
+                        const int i = first_own + o * kWGroups;
+                        const int32_t pp0 = it.q0 + k * kRawPlanes + i * kStagePp;
+                        const int32_t wd = pp0 % (kPosBlockSigned * p.planes_per_len) / kPosBlockSigned;
+#pragma unroll
+                        for (int c = 0; c < kWCols; ++c)
+                            sg_box[o][c] = i < ops_here ? __ldg(sign_col + (int64_t)wd * p.n_pad + c * (kUN / kWCols)) : make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
+                int own = 0;
                 site = 6;
                 ok = u_mbar_wait_warp(bar(kRawFull + s), (raw_cnt / kRawStages) & 1u, s_abort, lane);
                 if (!ok) break;
                 site = 8;
                 const uint32_t *raw_w = reinterpret_cast<const uint32_t *>(raw + (size_t)s * kRawStageBytes);
-                const int ops_here = min(kRawUnits, it.n_raw - k * kRawUnits) * kOpsPerRaw;    // units present in this box
                 for (int i = 0; i < ops_here; ++i, ++op_cnt) {
                     if ((int)(op_cnt % kWGroups) != group) continue;        // another group's stage
                     const uint32_t t = op_cnt % kOpStages;
                     // the bit words of this operand stage are read before the stage's buffer is awaited, so the
                     // shared-memory latency hides behind the wait
-                    constexpr int kStagePl = kOpSteps * kPpq;     // raw planes of one operand stage
+                    constexpr int kStagePl = kStagePp;            // raw planes of one operand stage
                     uint32_t pl[kWCols][kStagePl];
+                    uint4 sg[kWCols];
 #pragma unroll
                     for (int c = 0; c < kWCols; ++c) {
                         const int idx = row + c * (kUN / kWCols);
 #pragma unroll
                         for (int q = 0; q < kStagePl; ++q) pl[c][q] = raw_w[(i * kStagePl + q) * kUN + idx];
+                        if (kMode == SC_UNIPOLAR_AND) sg[c] = own == 0 ? sg_box[0][c] : sg_box[kOwnMax - 1][c];
                     }
+                    ++own;
                     // Use u of a stage waits for the MMAs of use u - 1.  Even and odd uses signal different barriers: a warp
                     // that fills only every third use of a stage would otherwise see the parity it waits for while the
                     // barrier is still two uses behind.
@@ -620,6 +673,8 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
 #pragma unroll
                     for (int c = 0; c < kWCols; ++c) {
                         uint8_t *op_b = ops + (size_t)t * kOpStageBytes + (row + c * (kUN / kWCols)) * 16;
+                        uint32_t sn[4] = {0u, 0u, 0u, 0u};
+                        if (kMode == SC_UNIPOLAR_AND) { sn[0] = sg[c].x; sn[1] = sg[c].y; sn[2] = sg[c].z; sn[3] = sg[c].w; }
 #pragma unroll
                         for (int st = 0; st < kOpSteps; ++st) {
                             uint32_t out[8];
@@ -627,8 +682,8 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
                                 u_expand_bits<true>(pl[c][2 * st], out);
                                 u_expand_bits<true>(pl[c][2 * st + 1], out + 4);
                             } else {
-                                u_expand_signed_w(pl[c][4 * st], pl[c][4 * st + 1], out);
-                                u_expand_signed_w(pl[c][4 * st + 2], pl[c][4 * st + 3], out + 4);
+                                u_expand_signed<true>(pl[c][2 * st], sn, out);
+                                u_expand_signed<true>(pl[c][2 * st + 1], sn, out + 4);
                             }
                             uint8_t *dst = op_b + 2u * st * kLboB;
                             *reinterpret_cast<uint4 *>(dst) = make_uint4(out[0], out[1], out[2], out[3]);
@@ -820,7 +875,10 @@ cudaError_t launch_core_umma(const CoreArgs &a, cudaStream_t st)
     UmmaDev dev;
     dev.a_streams = a.a_streams; dev.m_pad = a.m_pad;
     dev.perm = a.perm; dev.l_sorted = a.l_sorted; dev.plan = a.plan; dev.acc = a.acc; dev.scratch = a.scratch;
-    dev.N = a.N; dev.planes_per_len = a.kw * a.ppq;
+    dev.N = a.N; dev.planes_per_len = a.kw; dev.pos_block = a.pos_block;
+    dev.w_sign = a.w_sign; dev.a_sign = a.a_sign; dev.n_pad = a.n_pad;
+    if (a.mode == SC_UNIPOLAR_AND && (a.pos_block != kPosBlockSigned || !a.w_sign || !a.a_sign)) return cudaErrorInvalidValue;
+    if (a.mode != SC_UNIPOLAR_AND && a.pos_block != 1) return cudaErrorInvalidValue;
     dev.tiles_m = a.tiles_m; dev.w_batch_cols = a.w_batch_cols;
     if (a.mode == SC_UNIPOLAR_AND) return launch_umma_mode<SC_UNIPOLAR_AND>(mw, dev, a.sm_count, st);
     return launch_umma_mode<SC_BIPOLAR_XNOR>(mw, dev, a.sm_count, st);

@@ -91,15 +91,16 @@ SC_HD uint32_t sng_word(const PhiloxKeys &ks, uint32_t stream_word, uint64_t ele
 // Bipolar W planes: bit `lane` of a plane word holds depth element w_bit_element(lane) of the word's 32 elements (each
 // group of four in reverse order).
 SC_HD int w_bit_element(int lane) { return (lane & ~3) | (3 - (lane & 3)); }
-// Unipolar W planes: the two planes of a position as two-bit (stream bit, stream bit AND sign) fields: nibble j of p0
-// holds element 4 j at bits (2, 3) and element 4 j + 1 at bits (0, 1); p1 holds elements 4 j + 2 and 4 j + 3.
-SC_HD void pack_w_fields(uint32_t z, uint32_t n, uint32_t &p0, uint32_t &p1)
+// Unipolar (sign-magnitude) operands of the tensor-core core: one magnitude plane per position (W in that same reversed
+// order) plus, per (depth word, stream row), the signs of the 32 elements kept beside the planes -- a sign does not
+// depend on the position -- already spread into the four nibble words the expansion produces (sign_nibble_words).
+// Stream positions are stored in blocks: plane index of (position l, depth word w) with kw depth words and blocks of `block`
+// positions (1 = position-major, the plain layout).  With block = 8 the eight planes of one operand stage of the core
+// are eight positions of ONE depth word, so one set of sign words serves the whole stage.
+SC_HD int64_t plane_index(int32_t l, int32_t w, int32_t kw, int32_t block)
 {
-    const uint32_t m = 0x11111111u;
-    p0 = ((z >> 1) & m) | (((n >> 1) & m) << 1) | ((z & m) << 2) | ((n & m) << 3);
-    p1 = ((z >> 3) & m) | (((n >> 3) & m) << 1) | (((z >> 2) & m) << 2) | (((n >> 2) & m) << 3);
+    return (int64_t)(l / block) * kw * block + (int64_t)w * block + (l % block);
 }
-
 // Expansion, 1 stream bit -> one 4-bit float (e2m1: bit 3 sign, bits 2..0 = 0.5 / 1 / 2 for a single set bit).
 // 32 elements of a depth word become 32 nibbles = 4 words; nibble j of output word m <- element 4 j + m.
 //
@@ -123,27 +124,25 @@ SC_HD void u_expand_bits(uint32_t src, uint32_t out[4])
         out[3] = src & 0x11111111u;
     }
 }
-// Unipolar (sign-magnitude operands), activations: +-0.5 from the magnitude plane (value bit) and the negative plane
-// (sign bit).  Activations without any negative stream bit in the call skip the sign.
-SC_HD void u_expand_signed_a(uint32_t mag, uint32_t neg, uint32_t out[4], bool a_signed)
+// Unipolar (sign-magnitude operands): the same powers of two with the sign in bit 3 of the nibble, so every product is
+// +-1 and the accumulators hold the signed count.  s[m] has bit 3 of nibble j set iff element 4 j + m of the depth word
+// is negative (`sign_word`: bit b = sign of the element that sits at bit b of the plane words; W planes hold element m
+// of a nibble group at bit 3 - m, A planes at bit m).  A set sign on a zero magnitude is -0: harmless.
+SC_HD void sign_nibble_words(uint32_t sign_word, bool reversed, uint32_t s[4])
 {
 #if defined(__CUDA_ARCH__)
 #pragma unroll
 #endif
-    for (int m = 0; m < 4; ++m) {
-        out[m] = (mag >> m) & 0x11111111u;
-        if (a_signed) out[m] |= (neg << (3 - m)) & 0x88888888u;
-    }
+    for (int m = 0; m < 4; ++m) s[m] = (sign_word << (reversed ? m : 3 - m)) & 0x88888888u;
 }
-// Unipolar weights: +-2.  The encode stored each position as two planes of two-bit (stream bit, stream bit AND sign)
-// fields: nibble j of the first plane holds element 4 j at bits (2, 3) and element 4 j + 1 at bits (0, 1), the second
-// plane elements 4 j + 2 and 4 j + 3: one shift and one mask per output word.  Every product is +-1.
-SC_HD void u_expand_signed_w(uint32_t p0, uint32_t p1, uint32_t out[4])
+template <bool kHigh>
+SC_HD void u_expand_signed(uint32_t plane, const uint32_t s[4], uint32_t out[4])
 {
-    out[0] = p0 & 0xCCCCCCCCu;
-    out[1] = (p0 << 2) & 0xCCCCCCCCu;
-    out[2] = p1 & 0xCCCCCCCCu;
-    out[3] = (p1 << 2) & 0xCCCCCCCCu;
+    u_expand_bits<kHigh>(plane, out);
+#if defined(__CUDA_ARCH__)
+#pragma unroll
+#endif
+    for (int m = 0; m < 4; ++m) out[m] |= s[m];
 }
 
 #if defined(__CUDACC__)

@@ -4,6 +4,8 @@
 // Packed layout ("depth-packed planes"): plane p is a row of r_pad 32-bit words, one per stream row;
 // the word of stream row r in plane p = (l * kw + w) * ppq (+1 for the negative plane in unipolar
 // mode) holds stream position l of the 32 elements d = 32 w .. 32 w + 31 of that row (bit d % 32).
+// (The signed operands of the tensor-core core store the positions in blocks of 8, plane_index(l, w) * ppq, and
+// its unipolar W operand keeps one sign word per (w, stream row) beside single magnitude planes.)
 // The GEMM core then reduces over planes with whole-word XOR/AND + POPC, any integer length costs
 // exactly l * kw planes (no padding to a multiple of 32 positions), and a tile of 128 stream rows x
 // 16 planes is one 2-D TMA box.
@@ -28,6 +30,8 @@ struct EncodeDev {
     uint32_t *streams;
     int32_t *status;
     int32_t tensor_id, kw, Lmax, n_chunks, chunk_blocks, reverse_bytes, vec_rows, quant;
+    int32_t ppq, pos_block;          // planes per position written (unipolar: 2, or 1 when the signs go to `signs`); position blocks
+    uint32_t *signs;                 // [kw][r_pad][4] nibble sign words of a unipolar operand (NULL: negative planes instead)
     uint32_t stream_word;
     // weight operand of a batched call: stream row r = b * batch_pad + j is output column j of product b, stored at
     // X[b][d][j] (or X[b][j][d] when transposed); batch_pad = 0 otherwise
@@ -44,7 +48,6 @@ template <int kMode>
 __global__ void __launch_bounds__(kEncodeThreads)
 encode_kernel(const __grid_constant__ PhiloxKeys ks, const __grid_constant__ EncodeDev p)
 {
-    constexpr int kPpq = (kMode == SC_UNIPOLAR_AND) ? 2 : 1;
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (kEncodeThreads / 32) + (threadIdx.x >> 5);
     // warp index -> (row group, block run, depth word); depth word fastest so that neighbouring warps read
@@ -151,6 +154,18 @@ encode_kernel(const __grid_constant__ PhiloxKeys ks, const __grid_constant__ Enc
     // tensor-core core expand them with the cheap unsigned rule
     if (kMode == SC_UNIPOLAR_AND && p.tensor_id == 0 && any_negative && lane == 0) atomicOr(p.status + kSlotAnyNegA, 1);
 
+    // The tensor-core core takes the signs of a unipolar operand beside single magnitude planes: per (depth word, stream
+    // row) the four nibble sign words of the row's 32 elements.  The warp that owns the first run of blocks writes them
+    // (lane t the words of row t).
+    if (kMode == SC_UNIPOLAR_AND && p.signs && chunk == 0 && lane < 8) {
+        uint32_t sn[4];
+        uint32_t mine = neg_mask[0];
+#pragma unroll
+        for (int t = 1; t < 8; ++t) mine = lane == t ? neg_mask[t] : mine;
+        sign_nibble_words(mine, p.reverse_bytes == 1, sn);
+        reinterpret_cast<uint4 *>(p.signs)[(int64_t)w * p.r_pad + r0 + lane] = make_uint4(sn[0], sn[1], sn[2], sn[3]);
+    }
+
     // ---- phase 2: the blocks ----
 #pragma unroll 1
     for (int32_t blk = blk0; blk < blk1; ++blk) {
@@ -165,34 +180,17 @@ encode_kernel(const __grid_constant__ PhiloxKeys ks, const __grid_constant__ Enc
         }
         const int32_t l = blk * 32 + lane;                             // the position this lane holds
         if (l < l_write) {
-            const int64_t plane = ((int64_t)l * p.kw + w) * kPpq;
+            const int64_t plane = plane_index(l, w, p.kw, p.pos_block) * p.ppq;
             uint4 *dst = reinterpret_cast<uint4 *>(p.streams + plane * p.r_pad + r0);
-            if (kMode == SC_UNIPOLAR_AND && p.reverse_bytes == 2) {
-                // Two-bit (stream bit, stream bit AND sign) fields for the tensor-core core's signed weight operand:
-                // nibble j of the first plane holds element 4 j of the depth word at bits (2, 3) and element 4 j + 1 at
-                // bits (0, 1); the second plane holds elements 4 j + 2 and 4 j + 3 the same way.  One shift and one mask
-                // then turn a plane into eight signed 4-bit weights (+2 / -2 / 0).
-                uint32_t lo[8], hi[8];
-#pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    const uint32_t z = out_pos[t], n = out_pos[t] & neg_mask[t];
-                    pack_w_fields(z, n, lo[t], hi[t]);
-                }
+            dst[0] = make_uint4(out_pos[0], out_pos[1], out_pos[2], out_pos[3]);
+            dst[1] = make_uint4(out_pos[4], out_pos[5], out_pos[6], out_pos[7]);
+            if (kMode == SC_UNIPOLAR_AND && p.ppq == 2) {
+                // the negative plane: stream bit AND sign
                 uint4 *dn = reinterpret_cast<uint4 *>(p.streams + (plane + 1) * p.r_pad + r0);
-                dst[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-                dst[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
-                dn[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                dn[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-            } else {
-                dst[0] = make_uint4(out_pos[0], out_pos[1], out_pos[2], out_pos[3]);
-                dst[1] = make_uint4(out_pos[4], out_pos[5], out_pos[6], out_pos[7]);
-                if (kMode == SC_UNIPOLAR_AND) {
-                    uint4 *dn = reinterpret_cast<uint4 *>(p.streams + (plane + 1) * p.r_pad + r0);
-                    dn[0] = make_uint4(out_pos[0] & neg_mask[0], out_pos[1] & neg_mask[1], out_pos[2] & neg_mask[2],
-                                       out_pos[3] & neg_mask[3]);
-                    dn[1] = make_uint4(out_pos[4] & neg_mask[4], out_pos[5] & neg_mask[5], out_pos[6] & neg_mask[6],
-                                       out_pos[7] & neg_mask[7]);
-                }
+                dn[0] = make_uint4(out_pos[0] & neg_mask[0], out_pos[1] & neg_mask[1], out_pos[2] & neg_mask[2],
+                                   out_pos[3] & neg_mask[3]);
+                dn[1] = make_uint4(out_pos[4] & neg_mask[4], out_pos[5] & neg_mask[5], out_pos[6] & neg_mask[6],
+                                   out_pos[7] & neg_mask[7]);
             }
         }
     }
@@ -207,6 +205,8 @@ cudaError_t launch_encode(const EncodeArgs &a, cudaStream_t st)
     p.streams = a.streams; p.status = a.status;
     p.tensor_id = a.tensor_id; p.kw = (int32_t)a.kw; p.Lmax = a.Lmax; p.reverse_bytes = a.reverse_bytes;
     p.quant = a.quant;
+    p.pos_block = a.pos_block; p.signs = a.signs;
+    p.ppq = (a.mode == SC_UNIPOLAR_AND && !a.signs) ? 2 : 1;
     p.stream_word = ((uint32_t)a.tensor_id & 1u) | (a.stream_id << 1);
     p.batch_pad = a.batch_pad; p.batch_real = a.batch_real; p.w_transposed = a.w_transposed;
     // W read as two 16-byte vectors per lane when its rows keep them aligned

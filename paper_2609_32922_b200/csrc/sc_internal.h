@@ -51,6 +51,13 @@ long long launches_so_far();
 
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 inline int planes_per_step(int mode) { return mode == SC_UNIPOLAR_AND ? 2 : 1; }
+// Stream positions are stored in blocks of this many (plane_index in sc_device.cuh).  The signed (unipolar) operands of
+// the tensor-core core use blocks of 8, everything else the plain position-major order.
+constexpr int kPosBlockSigned = 8;
+inline int pos_block_for(int mode, bool umma) { return (umma && mode == SC_UNIPOLAR_AND) ? kPosBlockSigned : 1; }
+// planes per position as written for a core family: the tensor-core core keeps the signs of unipolar operands beside
+// single magnitude planes, the ALU cores read a magnitude and a negative plane
+inline int planes_per_step_for(int mode, bool umma) { return (umma || mode != SC_UNIPOLAR_AND) ? 1 : 2; }
 
 // Work plan written by the plan kernel and read by the core (device memory, int32 fields).
 struct PlanHeader {
@@ -75,8 +82,9 @@ struct BatchGeom {
 
 // Workspace offsets (bytes) of one sc_matmul call.
 struct Workspace {
-    size_t sigma_a, sigma_w, l_rows, perm, l_sorted, plan, acc, pop_a, pop_w, a_streams, w_streams, total;
-    int64_t m_pad, n_pad, kw, a_planes, w_planes;
+    size_t sigma_a, sigma_w, l_rows, perm, l_sorted, plan, acc, pop_a, pop_w, a_streams, w_streams, w_sign, a_sign, total;
+    int64_t m_pad, n_pad, kw, a_planes, w_planes;      // plane counts as allocated (unipolar: lengths rounded up to 8, two planes
+                                                       // per position for either core family)
 };
 // with_w = false leaves out everything derived from W alone (prepared weights carry it).
 Workspace layout_workspace(int64_t M, int64_t K, int64_t N, int32_t Lmax, int mode, bool need_acc, bool with_w = true,
@@ -84,7 +92,7 @@ Workspace layout_workspace(int64_t M, int64_t K, int64_t N, int32_t Lmax, int mo
 
 // Prepared weights: all that sc_matmul derives from W alone, kept in a caller-owned device buffer.
 struct WeightsLayout {
-    size_t sigma_w, pop_w, w_streams, total;
+    size_t sigma_w, pop_w, w_streams, w_sign, total;
     int64_t n_pad, kw, w_planes;
 };
 WeightsLayout layout_weights(int64_t K, int64_t N, int32_t Lmax, int mode);
@@ -101,6 +109,7 @@ struct sc_weights_impl {
     const float *sigma_w;
     const int32_t *pop_w;    // NULL unless umma && bipolar
     const uint32_t *w_streams;
+    const uint32_t *w_sign;  // NULL unless umma && unipolar
 };
 constexpr uint32_t kWeightsMagic = 0x53435754u;
 
@@ -127,7 +136,7 @@ cudaError_t launch_ladder_lengths(const float *g, int64_t M, int32_t group, cons
 cudaError_t launch_plan(const int32_t *L, int64_t M, int32_t group, int32_t Lmax, int64_t kw, int ppq,
                         int64_t m_pad, int64_t n_col_tiles, int32_t target_items, int32_t wave_ctas,
                         int32_t *l_rows, int32_t *perm, int32_t *l_sorted, PlanHeader *plan, int32_t *scratch,
-                        cudaStream_t st, int64_t batch = 1);
+                        cudaStream_t st, int64_t batch = 1, int32_t pos_block = 1);
 
 struct EncodeArgs {
     const float *X;
@@ -145,7 +154,10 @@ struct EncodeArgs {
     uint32_t *streams;
     int32_t *status;
     int reverse_bytes;           // W operand of the tensor-core core: 1 = each group of 4 depth elements in reverse bit
-                                 // order (bipolar), 2 = two-bit (stream bit, signed bit) fields (unipolar); 0 = plain
+                                 // order; 0 = plain
+    int pos_block = 1;           // stream positions stored in blocks of this many (plane_index)
+    uint32_t *signs = nullptr;   // unipolar operand of the tensor-core core: [kw][r_pad][4] nibble sign words written here
+                                 // and only the magnitude planes (one per position) into `streams`
     // W operand of a batched call (tensor_id 1): stream row r = b * batch_pad + j is output column j of product b
     int64_t batch_pad = 0;       // padded stream rows per product (0: not batched, rows = stream rows)
     int64_t batch_real = 0;      // real stream rows per product
@@ -171,6 +183,9 @@ struct CoreArgs {
     int32_t tiles_m = 1;         // row tiles per product and ...
     int64_t w_batch_cols = 0;    // ... padded W stream rows per product: the W tile of an item starts at
                                  // (row tile / tiles_m) * w_batch_cols + column tile * tile width
+    const uint32_t *w_sign = nullptr;   // unipolar tensor-core core: [kw][n_pad][4] nibble sign words of W ...
+    const uint32_t *a_sign = nullptr;   // ... and [kw][m_pad][4] of A (sorted row order)
+    int32_t pos_block = 1;       // block size of the stream positions in both operands' planes
     int32_t *pop_a;              // [M] ones of each row of A below its own end (tensor-core core, bipolar)
     const int32_t *pop_w;        // [(Lmax + 1) x n_pad] prefix ones of each W column (tensor-core core, bipolar)
 };

@@ -100,7 +100,7 @@ __device__ void finish_plan(int32_t n_row_tiles, int32_t n_col_tiles, int32_t ta
 // positions; source rows are numbered over all products (b * M + i).  A single product finishes the plan
 // in the same launch; several need plan_finish_kernel afterwards.
 __global__ void __launch_bounds__(kPlanThreads)
-plan_kernel(const int32_t *__restrict__ L, int64_t M, int32_t group, int32_t Lmax, int32_t planes_per_len,
+plan_kernel(const int32_t *__restrict__ L, int64_t M, int32_t group, int32_t Lmax, int32_t planes_per_len, int32_t pos_block,
             int64_t m_pad, int32_t n_col_tiles, int32_t target_items, int32_t wave_ctas,
             int32_t *__restrict__ l_rows,
             int32_t *__restrict__ perm, int32_t *__restrict__ l_sorted, PlanHeader *__restrict__ plan,
@@ -177,7 +177,8 @@ plan_kernel(const int32_t *__restrict__ L, int64_t M, int32_t group, int32_t Lma
     int32_t *prefix = reinterpret_cast<int32_t *>(plan + 1);
     int32_t *tile_planes = prefix + n_row_tiles + 1 + (int64_t)blockIdx.x * tiles_m;
     for (int32_t rt = tid; rt < tiles_m; rt += kPlanThreads)
-        tile_planes[rt] = l_sorted[(int64_t)rt * kTileM] * planes_per_len;        // longest row of the tile
+        // the longest row of the tile, in whole blocks of stream positions
+        tile_planes[rt] = (l_sorted[(int64_t)rt * kTileM] + pos_block - 1) / pos_block * pos_block * planes_per_len;
     __syncthreads();
     if (gridDim.x == 1) finish_plan(n_row_tiles, n_col_tiles, target_items, wave_ctas, planes_per_len, plan, scratch, s_cost, s_scan);
 }
@@ -194,10 +195,10 @@ plan_finish_kernel(int32_t n_row_tiles, int32_t n_col_tiles, int32_t target_item
 cudaError_t launch_plan(const int32_t *L, int64_t M, int32_t group, int32_t Lmax, int64_t kw, int ppq, int64_t m_pad,
                         int64_t n_col_tiles, int32_t target_items, int32_t wave_ctas, int32_t *l_rows,
                         int32_t *perm, int32_t *l_sorted, PlanHeader *plan, int32_t *scratch, cudaStream_t st,
-                        int64_t batch)
+                        int64_t batch, int32_t pos_block)
 {
     if (batch < 1 || batch > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
-    plan_kernel<<<(unsigned)batch, kPlanThreads, 0, st>>>(L, M, group, Lmax, (int32_t)(kw * ppq), m_pad, (int32_t)n_col_tiles,
+    plan_kernel<<<(unsigned)batch, kPlanThreads, 0, st>>>(L, M, group, Lmax, (int32_t)(kw * ppq), pos_block, m_pad, (int32_t)n_col_tiles,
                                                         target_items, wave_ctas, l_rows, perm, l_sorted, plan, scratch);
     count_launches(1);
     if (batch > 1) {
