@@ -58,7 +58,11 @@ typedef enum { SC_SCALE_NONE = 0,       /* sigma = 1, values are clamped to [-1,
 enum { SC_CORE_AUTO = 0, SC_CORE_POPC = 1,   /* LOP3 + POPC on the integer pipes                          */
        SC_CORE_CSA = 2,                      /* carry-save: 3 planes -> 2 POPC                             */
        SC_CORE_SIMPLE = 3,                   /* one thread per output, no staging (debug reference)        */
-       SC_CORE_UMMA = 4 };                   /* tcgen05 tensor cores (4-bit floats) on bits expanded on chip */
+       SC_CORE_UMMA = 4,                     /* tcgen05 tensor cores (4-bit floats) on bits expanded on chip,
+                                                one SM per 128 x 192 tile                                  */
+       SC_CORE_UMMA_PAIR = 5 };              /* the same on pairs of SMs (tcgen05 cta_group::2, 256 x 256 tiles); AUTO
+                                                picks between the two per call from the stream lengths (long work
+                                                pieces: pairs); batched calls always run on single SMs     */
 
 /* Value -> comparator boundary (sc_params.quant).  Sec. 4.2 maps operands to the int8 grid (q_max = 127) and then to
  * one of 257 comparison boundaries; how a grid point becomes a boundary is not printed. */

@@ -17,7 +17,7 @@ SC_OK, SC_ERR_ARG, SC_ERR_SHAPE, SC_ERR_LENGTH, SC_ERR_NONFINITE = 0, 1, 2, 3, 4
 SC_ERR_BUDGET, SC_ERR_WORKSPACE, SC_ERR_CUDA, SC_ERR_TIMEOUT = 5, 6, 7, 8
 SC_BIPOLAR_XNOR, SC_UNIPOLAR_AND = 0, 1
 SC_SCALE_NONE, SC_SCALE_PER_ROW, SC_SCALE_PER_TENSOR = 0, 1, 2
-SC_CORE_AUTO, SC_CORE_POPC, SC_CORE_CSA, SC_CORE_SIMPLE, SC_CORE_UMMA = 0, 1, 2, 3, 4
+SC_CORE_AUTO, SC_CORE_POPC, SC_CORE_CSA, SC_CORE_SIMPLE, SC_CORE_UMMA, SC_CORE_UMMA_PAIR = 0, 1, 2, 3, 4, 5
 SC_QUANT_DIRECT257, SC_QUANT_INT8_THEN_257 = 0, 1
 SC_L_CAP = 1024
 

@@ -77,6 +77,7 @@ static int pick_variant(const sc_params *p, int64_t K, int32_t Lmax)
 {
     const bool umma_fits = (int64_t)K * Lmax <= (1LL << 24);
     int variant = p->core == SC_CORE_AUTO ? (umma_fits ? SC_CORE_UMMA : SC_CORE_CSA) : (int)p->core;
+    if (variant == SC_CORE_UMMA_PAIR) variant = SC_CORE_UMMA;       // same family: one operand layout, two kernels
     if (variant == SC_CORE_UMMA && !umma_fits) variant = SC_CORE_CSA;
     return variant;
 }
@@ -89,7 +90,7 @@ static bool params_ok(const sc_params *p)
     if (p->scale_w < SC_SCALE_NONE || p->scale_w > SC_SCALE_PER_TENSOR) return false;
     if (p->group < 1) return false;
     if (p->stream_id >= (1u << 31)) return false;
-    if (p->core > SC_CORE_UMMA) return false;
+    if (p->core > SC_CORE_UMMA_PAIR) return false;
     if ((p->quant != SC_QUANT_DIRECT257 && p->quant != SC_QUANT_INT8_THEN_257) || p->reserved != 0) return false;
     return true;
 }
@@ -353,6 +354,15 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     const uint32_t *w_sign = pw ? pw->w_sign : w_sign_ws;
     uint32_t *a_sign = reinterpret_cast<uint32_t *>(base + w.a_sign);
     const bool signs = umma && params->mode == SC_UNIPOLAR_AND;
+    // The tensor-core family has two kernels: one SM per tile, and pairs of SMs.  AUTO lets the plan choose from the lengths
+    // (device data), an explicit request fixes it; batched calls and calls with too many row tiles stay on single SMs.
+    int pair_mode = 0, pair_clusters = 0;               // 0 never, 1 the plan decides, 2 always
+    if (umma && B == 1 && w.m_pad / kTileM <= pair_core_max_row_tiles() && params->core != SC_CORE_UMMA) {
+        pair_mode = params->core == SC_CORE_UMMA_PAIR ? 2 : 1;
+        if (pair_core_clusters(params->mode, c->sm_count, &pair_clusters) != cudaSuccess) return SC_ERR_CUDA;
+        if (pair_clusters < 1) pair_mode = 0;
+    }
+    const int32_t pair_col_tiles = (int32_t)((N + pair_core_tile_cols() - 1) / pair_core_tile_cols());
 
     auto mark = [&](int k) { if (c->profiling) cudaEventRecord(c->phase_ev[k], st); };
     c->profile_valid = false;
@@ -374,7 +384,8 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     // a3: row ordering by length and the work list
     auto plan_rows = [&]() -> bool {
         if (launch_plan(L, M, params->group, Lmax, w.kw, ppq, m_pad_b, n_col_tiles, umma ? 0 : c->sm_count * 16,
-                        umma ? c->sm_count : 0, l_rows, perm, l_sorted, plan, c->scratch, st, B, pos_block) != cudaSuccess)
+                        umma ? c->sm_count : 0, l_rows, perm, l_sorted, plan, c->scratch, st, B, pos_block, pair_col_tiles,
+                        pair_mode ? pair_clusters : 0, pair_mode == 2) != cudaSuccess)
             return false;
         // the W encode stops at the longest length of the call
         if (fork && (cudaEventRecord(c->ev_plan, st) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_plan, 0) != cudaSuccess))
@@ -439,7 +450,9 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     if (and_form && launch_row_corrections(ca, st) != cudaSuccess) return SC_ERR_CUDA;   // counted with the W encode phase
     mark(4);
     if (umma) {
+        // both kernels are enqueued; the one the plan did not select returns at once
         if (launch_core_umma(ca, st) != cudaSuccess) return SC_ERR_CUDA;
+        if (pair_mode && launch_core_umma_pair(ca, pair_clusters, pair_mode == 2, st) != cudaSuccess) return SC_ERR_CUDA;
     } else if (launch_core(ca, st) != cudaSuccess) {
         return SC_ERR_CUDA;
     }
@@ -666,7 +679,7 @@ sc_status sc_matmul_prepared(sc_ctx *ctx, const float *A, const sc_weights *weig
         return SC_ERR_ARG;
     if (Lmax > h->Lmax) return SC_ERR_LENGTH;
     // an explicit request for a core the buffer was not laid out for cannot be served
-    if (params->core != SC_CORE_AUTO && (params->core == SC_CORE_UMMA) != h->umma) return SC_ERR_ARG;
+    if (params->core != SC_CORE_AUTO && (params->core == SC_CORE_UMMA || params->core == SC_CORE_UMMA_PAIR) != h->umma) return SC_ERR_ARG;
     return matmul_impl(ctx, A, nullptr, h, M, h->K, h->N, L, Lmax, params, P, C, ws, ws_bytes, stream);
 }
 

@@ -66,7 +66,7 @@ struct PlanHeader {
     int32_t n_row_tiles;
     int32_t n_col_tiles;
     int32_t lmax_actual;
-    int32_t pad[3];
+    int32_t pad[3];         // pad[0]: 1 = the two-SM tensor-core core runs the call, 0 = the one-SM core
     // followed by int32 prefix[n_row_tiles + 1] and int32 tile_planes[n_row_tiles]
 };
 
@@ -136,7 +136,8 @@ cudaError_t launch_ladder_lengths(const float *g, int64_t M, int32_t group, cons
 cudaError_t launch_plan(const int32_t *L, int64_t M, int32_t group, int32_t Lmax, int64_t kw, int ppq,
                         int64_t m_pad, int64_t n_col_tiles, int32_t target_items, int32_t wave_ctas,
                         int32_t *l_rows, int32_t *perm, int32_t *l_sorted, PlanHeader *plan, int32_t *scratch,
-                        cudaStream_t st, int64_t batch = 1, int32_t pos_block = 1);
+                        cudaStream_t st, int64_t batch = 1, int32_t pos_block = 1, int32_t pair_col_tiles = 0,
+                        int32_t pair_clusters = 0, int32_t pair_force = 0);
 
 struct EncodeArgs {
     const float *X;
@@ -191,6 +192,12 @@ struct CoreArgs {
 };
 cudaError_t launch_core(const CoreArgs &a, cudaStream_t st);
 cudaError_t launch_core_umma(const CoreArgs &a, cudaStream_t st);
+// Two-SM tensor-core core (sc_core_umma2.cu): runs when the plan selected it (PlanHeader.pad[0]) or when forced; the one-SM
+// core returns at once in that case.  `clusters` = CTA pairs to launch (pair_core_clusters).
+cudaError_t launch_core_umma_pair(const CoreArgs &a, int clusters, bool force, cudaStream_t st);
+cudaError_t pair_core_clusters(int mode, int sm_count, int *clusters);
+int pair_core_tile_cols();
+int pair_core_max_row_tiles();
 cudaError_t launch_row_corrections(const CoreArgs &a, cudaStream_t st);
 cudaError_t launch_col_corrections(const uint32_t *w_streams, int64_t n_pad, int32_t kw, int32_t Lmax,
                                    const int32_t *lmax_actual, int32_t *pop_w, cudaStream_t st);

@@ -10,18 +10,47 @@ namespace sc {
 constexpr int kPlanThreads = 1024;
 
 // The work list over all row tiles (run by one CTA of kPlanThreads threads): chunk size, item prefix sums, totals.
+// Two-SM core (sc_core_umma2.cu): it has one accumulator, so a piece boundary drains its pipeline; it is selected when
+// the pieces are long -- min(mean stage units per piece, shortest tile pair) at least kPairMinUnits -- and its tiling of the
+// call (256 x 256 tiles on pairs of SMs; an odd row tile or a ragged last column tile is padding) costs no more MMA time
+// than the one-SM core's (128 x 192 tiles) after its measured advantage per multiply-accumulate on long pieces (7 %).
+constexpr int32_t kPairMinUnits = 96;
+constexpr long long kPairAdvantagePct = 107;
+
+struct PairChoice {
+    int32_t col_tiles;      // column tiles of the two-SM core (0: that core is not available for the call)
+    int32_t clusters;       // CTA pairs it runs with
+    int32_t force;          // select it whatever the lengths are
+};
+
 __device__ void finish_plan(int32_t n_row_tiles, int32_t n_col_tiles, int32_t target_items, int32_t wave_ctas,
                             int32_t planes_per_len, PlanHeader *__restrict__ plan, int32_t *scratch,
-                            unsigned long long *s_cost /* 64 */, int32_t *s_scan /* 34 */)
+                            unsigned long long *s_cost /* 64 */, int32_t *s_scan /* 34 */, PairChoice pair)
 {
+    __shared__ int32_t s_pair_min;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t *prefix = reinterpret_cast<int32_t *>(plan + 1);
     int32_t *tile_planes = prefix + n_row_tiles + 1;
     int32_t *s_max = s_scan + 32, *s_chunk = s_scan + 33;
     // the longest tile (tile 0 of the product with the longest row) and, for the ALU cores, the total work
     if (tid < 64) s_cost[tid] = 0ull;
-    if (tid == 0) *s_max = 0;
+    if (tid == 0) { *s_max = 0; s_pair_min = 0x7FFFFFFF; }
     __syncthreads();
+    if (pair.clusters > 0) {
+        // stage units of the row-tile pairs (the first, longer tile of a pair decides) per column tile of that core
+        unsigned long long units = 0, with_work = 0, single_units = 0;
+        int32_t shortest = 0x7FFFFFFF;
+        for (int32_t T = tid; 2 * T < n_row_tiles; T += kPlanThreads) {
+            const int32_t u = (tile_planes[2 * T] + kStagePlanes - 1) / kStagePlanes;
+            if (u > 0) { units += (unsigned long long)u; ++with_work; shortest = min(shortest, u); }
+            single_units += (unsigned long long)u;
+            if (2 * T + 1 < n_row_tiles) single_units += (unsigned long long)((tile_planes[2 * T + 1] + kStagePlanes - 1) / kStagePlanes);
+        }
+        if (with_work) {
+            atomicAdd(&s_cost[1], units); atomicAdd(&s_cost[2], with_work); atomicAdd(&s_cost[3], single_units);
+            atomicMin(&s_pair_min, shortest);
+        }
+    }
     int32_t mine = 0;
     unsigned long long work = 0;
     for (int32_t rt = tid; rt < n_row_tiles; rt += kPlanThreads) {
@@ -90,6 +119,17 @@ __device__ void finish_plan(int32_t n_row_tiles, int32_t n_col_tiles, int32_t ta
         plan->n_row_tiles = n_row_tiles;
         plan->n_col_tiles = n_col_tiles;
         plan->lmax_actual = longest / planes_per_len;
+        int32_t use_pair = 0;
+        if (pair.clusters > 0 && s_cost[2] > 0) {
+            const long long pieces = (long long)s_cost[2] * pair.col_tiles + pair.clusters;
+            const long long mean = (long long)s_cost[1] * pair.col_tiles / pieces;
+            // MMA time of the two tilings, up to a common factor: units x column tiles x tile columns / SMs per tile
+            const long long t_pair = (long long)s_cost[1] * pair.col_tiles * 256 * 2;
+            const long long t_single = (long long)s_cost[3] * n_col_tiles * kTileNUmma;
+            use_pair = (pair.force || (min(mean, (long long)s_pair_min) >= kPairMinUnits &&
+                                       t_pair * 100 <= t_single * kPairAdvantagePct)) ? 1 : 0;
+        }
+        plan->pad[0] = use_pair;                      // which tensor-core core runs: 1 = the two-SM core
         scratch[kSlotTicket] = 0;
         scratch[kSlotAnyNegA] = 0;                    // the encode of A sets it again if it meets a negative element
         scratch[kSlotLmaxActual] = longest / planes_per_len;
@@ -104,7 +144,7 @@ plan_kernel(const int32_t *__restrict__ L, int64_t M, int32_t group, int32_t Lma
             int64_t m_pad, int32_t n_col_tiles, int32_t target_items, int32_t wave_ctas,
             int32_t *__restrict__ l_rows,
             int32_t *__restrict__ perm, int32_t *__restrict__ l_sorted, PlanHeader *__restrict__ plan,
-            int32_t *scratch)
+            int32_t *scratch, PairChoice pair)
 {
     __shared__ int32_t bins[SC_L_CAP + 1];       // bins[v]: rows with length v, then running offsets
     __shared__ int32_t warp_sums[32];
@@ -180,7 +220,7 @@ plan_kernel(const int32_t *__restrict__ L, int64_t M, int32_t group, int32_t Lma
         // the longest row of the tile, in whole blocks of stream positions
         tile_planes[rt] = (l_sorted[(int64_t)rt * kTileM] + pos_block - 1) / pos_block * pos_block * planes_per_len;
     __syncthreads();
-    if (gridDim.x == 1) finish_plan(n_row_tiles, n_col_tiles, target_items, wave_ctas, planes_per_len, plan, scratch, s_cost, s_scan);
+    if (gridDim.x == 1) finish_plan(n_row_tiles, n_col_tiles, target_items, wave_ctas, planes_per_len, plan, scratch, s_cost, s_scan, pair);
 }
 
 __global__ void __launch_bounds__(kPlanThreads)
@@ -189,17 +229,18 @@ plan_finish_kernel(int32_t n_row_tiles, int32_t n_col_tiles, int32_t target_item
 {
     __shared__ unsigned long long s_cost[64];
     __shared__ int32_t s_scan[34];
-    finish_plan(n_row_tiles, n_col_tiles, target_items, wave_ctas, planes_per_len, plan, scratch, s_cost, s_scan);
+    finish_plan(n_row_tiles, n_col_tiles, target_items, wave_ctas, planes_per_len, plan, scratch, s_cost, s_scan, PairChoice{0, 0, 0});
 }
 
 cudaError_t launch_plan(const int32_t *L, int64_t M, int32_t group, int32_t Lmax, int64_t kw, int ppq, int64_t m_pad,
                         int64_t n_col_tiles, int32_t target_items, int32_t wave_ctas, int32_t *l_rows,
                         int32_t *perm, int32_t *l_sorted, PlanHeader *plan, int32_t *scratch, cudaStream_t st,
-                        int64_t batch, int32_t pos_block)
+                        int64_t batch, int32_t pos_block, int32_t pair_col_tiles, int32_t pair_clusters, int32_t pair_force)
 {
+    const PairChoice pair{pair_col_tiles, batch == 1 ? pair_clusters : 0, pair_force};
     if (batch < 1 || batch > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
     plan_kernel<<<(unsigned)batch, kPlanThreads, 0, st>>>(L, M, group, Lmax, (int32_t)(kw * ppq), pos_block, m_pad, (int32_t)n_col_tiles,
-                                                        target_items, wave_ctas, l_rows, perm, l_sorted, plan, scratch);
+                                                        target_items, wave_ctas, l_rows, perm, l_sorted, plan, scratch, pair);
     count_launches(1);
     if (batch > 1) {
         plan_finish_kernel<<<1, kPlanThreads, 0, st>>>((int32_t)(batch * (m_pad / kTileM)), (int32_t)n_col_tiles, target_items,

@@ -26,14 +26,14 @@ def sc(binding):
     s.close()
 
 
-@pytest.mark.parametrize("case", range(24))
+@pytest.mark.parametrize("case", range(30))
 def test_random_single_products(sc, binding, oracle, case):
     import torch
     rng = np.random.default_rng(1000 + case)
     M, K, N = int(rng.integers(1, 300)), int(rng.integers(1, 200)), int(rng.integers(1, 420))
     Lmax = int(rng.choice([1, 7, 32, 33, 64, 100]))
     mode = ["bipolar", "unipolar"][case % 2]
-    core = [0, 1, 2, 3, 4][case % 5]
+    core = [0, 1, 2, 3, 4, 5][case % 6] if case < 24 else 5
     group = int(rng.choice([1, 1, 3, 8]))
     w, _ = wl.small_ragged(seed=case, M=M, K=K, N=N, mode=mode, Lmax=Lmax)
     w = dataclasses.replace(w, scale_a=str(rng.choice(["none", "per_row", "per_tensor"])),

@@ -28,7 +28,7 @@ def sc(binding):
     s.close()
 
 
-CORES = [1, 2, 3, 4]   # POPC, carry-save, simple, tensor-core
+CORES = [1, 2, 3, 4, 5]   # POPC, carry-save, simple, tensor-core (one SM per tile), tensor-core (pairs of SMs)
 
 
 def test_row_stats_and_scales(sc, binding, oracle):
@@ -202,7 +202,7 @@ def _sampled_parity(sc, binding, oracle, w, A, W, L_groups, Lmax, group, n_rows,
     return P, C, L_rows
 
 
-@pytest.mark.parametrize("core", [1, 2, 4])
+@pytest.mark.parametrize("core", [1, 2, 4, 5])
 def test_config2_vit_b_fc1_sampled(sc, binding, oracle, core):
     w = wl.VIT_B_FC1
     A, W = wl.make_inputs(w)
@@ -216,7 +216,7 @@ def test_config2_vit_b_fc1_sampled(sc, binding, oracle, core):
     assert abs(z.mean()) < 0.01 and 0.5 < z.std() < 1.05
 
 
-@pytest.mark.parametrize("core", [0, 4])
+@pytest.mark.parametrize("core", [0, 4, 5])
 def test_config3_mixed_precision_sampled(sc, binding, oracle, core):
     w = wl.VIT_B_QKV_MIXED
     A, W = wl.make_inputs(w)
@@ -225,7 +225,7 @@ def test_config3_mixed_precision_sampled(sc, binding, oracle, core):
     _sampled_parity(sc, binding, oracle, w, A, W, L_groups, 256, 1, 24, 40, core=core)
 
 
-@pytest.mark.parametrize("core", [0, 4])
+@pytest.mark.parametrize("core", [0, 4, 5])
 def test_config4_dit_grouped_sampled(sc, binding, oracle, core):
     w = wl.DIT_XL_LINEAR
     A, W = wl.make_inputs(w)
@@ -336,8 +336,9 @@ def test_tensor_core_headroom_fallback(sc, binding, oracle, core):
     assert np.array_equal(P, ref["P"]) and T.close_enough(C, ref["C"])
 
 
+@pytest.mark.parametrize("core", [4, 5])
 @pytest.mark.parametrize("mode", ["bipolar", "unipolar"])
-def test_tensor_core_counts_exact_at_the_headroom_limit(sc, binding, mode):
+def test_tensor_core_counts_exact_at_the_headroom_limit(sc, binding, mode, core):
     """K * Lmax = 2^24 exactly, operands at +-1 so that every stream bit is known in closed form (a value of +1 is the
     all-ones stream; -1 is all zeros in bipolar mode and all ones with a negative sign in unipolar mode).  The counts
     reach 2^24 (bipolar) or +-2^23 (unipolar): the largest sums the tensor-core core's fp32 accumulators must hold exactly."""
@@ -351,7 +352,7 @@ def test_tensor_core_counts_exact_at_the_headroom_limit(sc, binding, mode):
     A[1::3, : K // 4] = -1.0              # every third row: the first quarter of the depth at -1
     L_rows = np.full(M, L, dtype=np.int32)
     L_rows[5] = 1000
-    P, C = T.gpu_matmul(sc, binding, w, A, W, L_rows, L, core=4)
+    P, C = T.gpu_matmul(sc, binding, w, A, W, L_rows, L, core=core)
     # signs: s_a[i][d] * s_w[d][j] summed over d, per position
     sa = np.where(A < 0, -1, 1).astype(np.int64)
     sw = np.where(W < 0, -1, 1).astype(np.int64)
@@ -432,10 +433,10 @@ def test_cores_agree_on_every_output_and_repeat(sc, binding, oracle, name):
     dA, dW = torch.from_numpy(A).cuda(), torch.from_numpy(W).cuda()
     dL = None if L_groups is None else torch.from_numpy(np.ascontiguousarray(L_groups, dtype=np.int32)).cuda()
     outs = []
-    for core in (4, 4, 2):
+    for core in (4, 4, 2, 5, 5, 0):
         P, C = sc.matmul(dA, dW, dL, Lmax, T.gpu_params(binding, w, group, core))
         torch.cuda.synchronize()
         outs.append((P.clone(), C.clone()))
-    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
-    assert torch.equal(outs[0][0], outs[2][0])
-    assert torch.equal(outs[0][1], outs[2][1])          # same decode arithmetic on the same counts
+    for k in range(1, len(outs)):                       # one-SM tensor core twice, carry-save, SM pairs twice, automatic choice
+        assert torch.equal(outs[0][0], outs[k][0]), k
+        assert torch.equal(outs[0][1], outs[k][1]), k   # same decode arithmetic on the same counts
