@@ -43,7 +43,6 @@ constexpr int kPWFirstWarp = kPAFirstWarp + kPAGroups * kPAWarps;
 constexpr int kPIssuers = 3;
 constexpr int kPIssuerBWarp = kPWFirstWarp + kPWGroups * kPWWarps;
 constexpr int kPThreads = 32 * (kPIssuerBWarp + kPIssuers - 1);
-constexpr int kPFillArrivals = 2 * (kPAWarps + kPWWarps);      // arrivals per operand stage: the expander warps of both CTAs
 static_assert(kPOpStages % kPIssuers == 0 && kPOpStages % kPAGroups == 0 && kPOpStages % kPWGroups == 0,
               "issuers and expander groups own fixed ring slots");
 static_assert(kPAFirstWarp % 4 == 2 && kPAWarps == 4 && kPStagePp == kPosBlockSigned && kPThreads <= 1024, "role layout");
@@ -59,9 +58,11 @@ constexpr uint32_t kPSfCol = 448, kPSfCols = 64;                // scale factors
 static_assert(kPARingCol + kPOpStages * kPOpSteps * 8 <= kPSfCol && kPSfCol + kPSfCols == kPTmemCols, "tensor memory budget");
 constexpr int kPMaxPairs = 1024;                                // row-tile pairs whose unit prefix fits the shared-memory table
 
+// "stage full" is four barriers per ring slot -- the activation and the weight expanders of either CTA arrive on a
+// barrier of their own, the issuer awaits all four -- because arrivals on one barrier are served one after another.
 enum PBar : int {
     kPRawFull = 0, kPRawEmpty = kPRawFull + kPRawStages, kPOpFull = kPRawEmpty + kPRawStages,
-    kPOpEmpty = kPOpFull + kPOpStages, kPAccFull = kPOpEmpty + 2 * kPOpStages, kPAccEmpty = kPAccFull + 1,
+    kPOpEmpty = kPOpFull + 4 * kPOpStages, kPAccFull = kPOpEmpty + 2 * kPOpStages, kPAccEmpty = kPAccFull + 1,
     kPAccStarted = kPAccEmpty + 1, kPNumBars = kPAccStarted + 1
 };
 constexpr size_t kPairSmem = (size_t)kPRawStages * kPRawStageBytes + (size_t)kPOpStages * kPOpStageBytes + kPEpiBytes +
@@ -197,7 +198,8 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
 
     if (tid == 0) {
         for (int s = 0; s < kPRawStages; ++s) { u_mbar_init(bar(kPRawFull + s), 1); u_mbar_init(bar(kPRawEmpty + s), kPWGroups * kPWWarps); }
-        for (int s = 0; s < kPOpStages; ++s) u_mbar_init(bar(kPOpFull + s), kPFillArrivals);
+        for (int s = 0; s < kPOpStages; ++s)
+            for (int k = 0; k < 4; ++k) u_mbar_init(bar(kPOpFull + 4 * s + k), k < 2 ? kPAWarps : kPWWarps);
         for (int s = 0; s < 2 * kPOpStages; ++s) u_mbar_init(bar(kPOpEmpty + s), 1);
         u_mbar_init(bar(kPAccFull), kPIssuers);
         u_mbar_init(bar(kPAccEmpty), 2 * kPEpiWarps);
@@ -306,7 +308,8 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
                 for (int32_t j = 0; j < n_ops; ++j, ++op_cnt) {
                     if (op_cnt % kPIssuers != me) continue;
                     const uint32_t t = op_cnt % kPOpStages;
-                    ok = p_mbar_wait_cluster(bar(kPOpFull + t), (op_cnt / kPOpStages) & 1u, s_abort);
+                    for (int k = 0; k < 4 && ok; ++k)
+                        ok = p_mbar_wait_cluster(bar(kPOpFull + 4 * t + k), (op_cnt / kPOpStages) & 1u, s_abort);
                     if (!ok) break;
                     u_fence_after();
                     const uint64_t bdesc = desc0 + (uint64_t)(t * kStageDesc);
@@ -477,7 +480,7 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 u_fence_before();
                 __syncwarp();
-                if (lane == 0) p_arrive_cta(bar(kPOpFull + t), 0u);
+                if (lane == 0) p_arrive_cta(bar(kPOpFull + 4 * t + rank), 0u);
             };
             AIter it;
             it.pos = run0; it.op = 0u;
@@ -587,7 +590,7 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA
                     __syncwarp();
-                    if (lane == 0) p_arrive_cta(bar(kPOpFull + t), 0u);
+                    if (lane == 0) p_arrive_cta(bar(kPOpFull + 4 * t + 2 + rank), 0u);
                 }
                 if (!ok) break;
                 __syncwarp();
