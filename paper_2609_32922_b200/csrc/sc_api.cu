@@ -363,6 +363,15 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
         if (pair_clusters < 1) pair_mode = 0;
     }
     const int32_t pair_col_tiles = (int32_t)((N + pair_core_tile_cols() - 1) / pair_core_tile_cols());
+    if (pair_mode == 1) {
+        // The plan selects the two-SM core only if its tiling costs at most 7 % more MMA time than the one-SM core's (its
+        // measured advantage on long pieces).  Where the shape alone already rules that out (an odd row tile, a ragged last
+        // column tile: ragged lengths only add to it), the two-SM kernel is not enqueued at all.
+        const int64_t row_tiles = w.m_pad / kTileM, pairs = (row_tiles + 1) / 2;
+        const int64_t t_pair = pairs * pair_col_tiles * pair_core_tile_cols() * 2;
+        const int64_t t_single = row_tiles * ((N + kTileNUmma - 1) / kTileNUmma) * kTileNUmma;
+        if (t_pair * 100 > t_single * 107) pair_mode = 0;
+    }
 
     auto mark = [&](int k) { if (c->profiling) cudaEventRecord(c->phase_ev[k], st); };
     c->profile_valid = false;
@@ -798,6 +807,7 @@ int32_t sc_selftest_expansion(void)
                     const int64_t pi = plane_index(l, w, 5, kPosBlockSigned);
                     if (pi < 0 || pi >= 24 * 5 || seen[pi]) ++mismatches; else seen[pi] = true;
                     if (plane_index(l, w, 5, 1) != (int64_t)l * 5 + w) ++mismatches;
+                    if (plane_index_pow2(l, w, 5, 3) != pi || plane_index_pow2(l, w, 5, 0) != (int64_t)l * 5 + w) ++mismatches;
                 }
         }
     }

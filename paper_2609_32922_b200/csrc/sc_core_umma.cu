@@ -431,7 +431,7 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
             // stage these are the leading ones: position-major, the pairs below l_i * (depth words); in blocks of 8
             // positions, the stage is positions lb .. lb + 7 of one depth word.
             int32_t n_act;
-            if (p.pos_block == 1) n_act = min(x.my_len * p.planes_per_len, x.q1) - pp0;
+            if (kMode == SC_BIPOLAR_XNOR) n_act = min(x.my_len * p.planes_per_len, x.q1) - pp0;
             else n_act = min(x.my_len - pp0 / (kPosBlockSigned * p.planes_per_len) * kPosBlockSigned, x.q1 - pp0);
             const uint32_t *src = p.a_streams + (int64_t)pp0 * p.m_pad + (int64_t)x.rt * kTileM + row;
 #pragma unroll

@@ -101,6 +101,11 @@ SC_HD int64_t plane_index(int32_t l, int32_t w, int32_t kw, int32_t block)
 {
     return (int64_t)(l / block) * kw * block + (int64_t)w * block + (l % block);
 }
+// the same for block = 2^shift, without a division
+SC_HD int64_t plane_index_pow2(int32_t l, int32_t w, int32_t kw, int32_t shift)
+{
+    return ((((int64_t)(l >> shift) * kw + w)) << shift) + (l & ((1 << shift) - 1));
+}
 // Expansion, 1 stream bit -> one 4-bit float (e2m1: bit 3 sign, bits 2..0 = 0.5 / 1 / 2 for a single set bit).
 // 32 elements of a depth word become 32 nibbles = 4 words; nibble j of output word m <- element 4 j + m.
 //

@@ -30,7 +30,7 @@ struct EncodeDev {
     uint32_t *streams;
     int32_t *status;
     int32_t tensor_id, kw, Lmax, n_chunks, chunk_blocks, reverse_bytes, vec_rows, quant;
-    int32_t ppq, pos_block;          // planes per position written (unipolar: 2, or 1 when the signs go to `signs`); position blocks
+    int32_t ppq, pos_shift;          // planes per position written (unipolar: 2, or 1 when the signs go to `signs`); log2 of the position block
     uint32_t *signs;                 // [kw][r_pad][4] nibble sign words of a unipolar operand (NULL: negative planes instead)
     uint32_t stream_word;
     // weight operand of a batched call: stream row r = b * batch_pad + j is output column j of product b, stored at
@@ -180,7 +180,7 @@ encode_kernel(const __grid_constant__ PhiloxKeys ks, const __grid_constant__ Enc
         }
         const int32_t l = blk * 32 + lane;                             // the position this lane holds
         if (l < l_write) {
-            const int64_t plane = plane_index(l, w, p.kw, p.pos_block) * p.ppq;
+            const int64_t plane = plane_index_pow2(l, w, p.kw, p.pos_shift) * p.ppq;
             uint4 *dst = reinterpret_cast<uint4 *>(p.streams + plane * p.r_pad + r0);
             dst[0] = make_uint4(out_pos[0], out_pos[1], out_pos[2], out_pos[3]);
             dst[1] = make_uint4(out_pos[4], out_pos[5], out_pos[6], out_pos[7]);
@@ -205,7 +205,8 @@ cudaError_t launch_encode(const EncodeArgs &a, cudaStream_t st)
     p.streams = a.streams; p.status = a.status;
     p.tensor_id = a.tensor_id; p.kw = (int32_t)a.kw; p.Lmax = a.Lmax; p.reverse_bytes = a.reverse_bytes;
     p.quant = a.quant;
-    p.pos_block = a.pos_block; p.signs = a.signs;
+    p.pos_shift = a.pos_block == kPosBlockSigned ? 3 : 0; p.signs = a.signs;
+    if (a.pos_block != 1 && a.pos_block != kPosBlockSigned) return cudaErrorInvalidValue;
     p.ppq = (a.mode == SC_UNIPOLAR_AND && !a.signs) ? 2 : 1;
     p.stream_word = ((uint32_t)a.tensor_id & 1u) | (a.stream_id << 1);
     p.batch_pad = a.batch_pad; p.batch_real = a.batch_real; p.w_transposed = a.w_transposed;
