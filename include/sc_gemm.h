@@ -217,7 +217,7 @@ sc_status sc_matmul_prepared(sc_ctx *ctx, const float *A, const sc_weights *weig
  * recovered exactly.  The paper leaves open which Sobol dimensions, scrambling and gating order its kernel uses:
  * here activation = dimension 1, weight generators = dimension 2, each XORed with a byte derived from
  * (seed, stream_id); comparator z = [r < T], boundaries as in sc_matmul (bipolar).
- * Arguments as sc_matmul, with: mode must be SC_BIPOLAR_XNOR, core SC_CORE_AUTO or SC_CORE_UMMA (the product
+ * Arguments as sc_matmul, with: mode must be SC_BIPOLAR_XNOR, core SC_CORE_AUTO, SC_CORE_UMMA or SC_CORE_UMMA_PAIR (the product
  * runs on the tensor-core core as a binary contraction of codes of 2 L_i positions per element of row i, so
  * its cost follows the sum of the lengths), 1 <= Lmax <= 256, 2 K Lmax <= 2^24.  P receives the XNOR counts of
  * the cycle-by-cycle multiplier.  Workspace: sc_workspace_bytes_cbsg(M, K, N, Lmax, params).            */

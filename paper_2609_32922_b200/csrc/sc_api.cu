@@ -95,6 +95,34 @@ static bool params_ok(const sc_params *p)
     return true;
 }
 
+// The tensor-core family has two kernels: one SM per tile, and pairs of SMs.  AUTO lets the plan choose from the lengths
+// (device data), an explicit request fixes it; batched calls and calls with too many row tiles stay on single SMs.
+struct PairLaunch {
+    int mode;               // 0 never (the two-SM kernel is not enqueued), 1 the plan decides, 2 always
+    int clusters;           // CTA pairs the two-SM kernel runs with
+    int32_t col_tiles;      // its column tiles
+};
+static bool choose_pair(sc_ctx_impl *c, const sc_params *params, bool umma, int64_t m_pad, int64_t N, int64_t B, PairLaunch *out)
+{
+    out->mode = 0;
+    out->clusters = 0;
+    out->col_tiles = (int32_t)((N + pair_core_tile_cols() - 1) / pair_core_tile_cols());
+    if (!umma || B != 1 || m_pad / kTileM > pair_core_max_row_tiles() || params->core == SC_CORE_UMMA) return true;
+    out->mode = params->core == SC_CORE_UMMA_PAIR ? 2 : 1;
+    if (pair_core_clusters(params->mode, c->sm_count, &out->clusters) != cudaSuccess) return false;
+    if (out->clusters < 1) out->mode = 0;
+    if (out->mode == 1) {
+        // The plan selects the two-SM core only if its tiling costs at most 7 % more MMA time than the one-SM core's (its
+        // measured advantage on long pieces).  Where the shape alone already rules that out (an odd row tile, a ragged last
+        // column tile: ragged lengths only add to it), the two-SM kernel is not enqueued at all.
+        const int64_t row_tiles = m_pad / kTileM, pairs = (row_tiles + 1) / 2;
+        const int64_t t_pair = pairs * out->col_tiles * pair_core_tile_cols() * 2;
+        const int64_t t_single = row_tiles * ((N + kTileNUmma - 1) / kTileNUmma) * kTileNUmma;
+        if (t_pair * 100 > t_single * 107) out->mode = 0;
+    }
+    return true;
+}
+
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // sigma of one operand into `sigma` (one entry per stream row)
@@ -354,24 +382,10 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     const uint32_t *w_sign = pw ? pw->w_sign : w_sign_ws;
     uint32_t *a_sign = reinterpret_cast<uint32_t *>(base + w.a_sign);
     const bool signs = umma && params->mode == SC_UNIPOLAR_AND;
-    // The tensor-core family has two kernels: one SM per tile, and pairs of SMs.  AUTO lets the plan choose from the lengths
-    // (device data), an explicit request fixes it; batched calls and calls with too many row tiles stay on single SMs.
-    int pair_mode = 0, pair_clusters = 0;               // 0 never, 1 the plan decides, 2 always
-    if (umma && B == 1 && w.m_pad / kTileM <= pair_core_max_row_tiles() && params->core != SC_CORE_UMMA) {
-        pair_mode = params->core == SC_CORE_UMMA_PAIR ? 2 : 1;
-        if (pair_core_clusters(params->mode, c->sm_count, &pair_clusters) != cudaSuccess) return SC_ERR_CUDA;
-        if (pair_clusters < 1) pair_mode = 0;
-    }
-    const int32_t pair_col_tiles = (int32_t)((N + pair_core_tile_cols() - 1) / pair_core_tile_cols());
-    if (pair_mode == 1) {
-        // The plan selects the two-SM core only if its tiling costs at most 7 % more MMA time than the one-SM core's (its
-        // measured advantage on long pieces).  Where the shape alone already rules that out (an odd row tile, a ragged last
-        // column tile: ragged lengths only add to it), the two-SM kernel is not enqueued at all.
-        const int64_t row_tiles = w.m_pad / kTileM, pairs = (row_tiles + 1) / 2;
-        const int64_t t_pair = pairs * pair_col_tiles * pair_core_tile_cols() * 2;
-        const int64_t t_single = row_tiles * ((N + kTileNUmma - 1) / kTileNUmma) * kTileNUmma;
-        if (t_pair * 100 > t_single * 107) pair_mode = 0;
-    }
+    PairLaunch pair;
+    if (!choose_pair(c, params, umma, w.m_pad, N, B, &pair)) return SC_ERR_CUDA;
+    const int pair_mode = pair.mode, pair_clusters = pair.clusters;
+    const int32_t pair_col_tiles = pair.col_tiles;
 
     auto mark = [&](int k) { if (c->profiling) cudaEventRecord(c->phase_ev[k], st); };
     c->profile_valid = false;
@@ -506,7 +520,7 @@ sc_status sc_matmul_batched(sc_ctx *ctx, const float *A, const float *W, int64_t
 static bool cbsg_args_ok(const sc_params *p, int64_t M, int64_t K, int64_t N)
 {
     if (!params_ok(p) || p->mode != SC_BIPOLAR_XNOR) return false;
-    if (p->core != SC_CORE_AUTO && p->core != SC_CORE_UMMA) return false;
+    if (p->core != SC_CORE_AUTO && p->core != SC_CORE_UMMA && p->core != SC_CORE_UMMA_PAIR) return false;
     return M > 0 && K > 0 && N > 0;
 }
 
@@ -557,8 +571,11 @@ sc_status sc_matmul_cbsg(sc_ctx *ctx, const float *A, const float *W, int64_t M,
     if (launch_cbsg_setup(params->seed, params->stream_id, tables, L, n_groups, Lmax, l_core, status, st) != cudaSuccess)
         return SC_ERR_CUDA;
     const int64_t n_col_tiles = (N + kTileNUmma - 1) / kTileNUmma;
+    PairLaunch pair;
+    if (!choose_pair(c, params, true, w.m_pad, N, 1, &pair)) return SC_ERR_CUDA;
     if (launch_plan(l_core, M, params->group, core_lmax, w.kw, 1, w.m_pad, n_col_tiles, 0, c->sm_count, l_rows,
-                    perm, l_sorted, plan, c->scratch, st) != cudaSuccess)
+                    perm, l_sorted, plan, c->scratch, st, 1, 1, pair.col_tiles, pair.mode ? pair.clusters : 0,
+                    pair.mode == 2) != cudaSuccess)
         return SC_ERR_CUDA;
     if (cudaMemsetAsync(acc, 0, sizeof(int32_t) * (size_t)M * (size_t)N, st) != cudaSuccess) return SC_ERR_CUDA;
     mark(2);
@@ -579,6 +596,7 @@ sc_status sc_matmul_cbsg(sc_ctx *ctx, const float *A, const float *W, int64_t M,
     ca.acc = acc; ca.scratch = c->scratch; ca.sm_count = c->sm_count; ca.Lmax = core_lmax;
     ca.pop_a = nullptr; ca.pop_w = nullptr;
     if (launch_core_umma(ca, st) != cudaSuccess) return SC_ERR_CUDA;
+    if (pair.mode && launch_core_umma_pair(ca, pair.clusters, pair.mode == 2, st) != cudaSuccess) return SC_ERR_CUDA;
     mark(5);
     if (launch_cbsg_decode(acc, M, N, K, L, params->group, Lmax, sigma_a, sigma_w, P, C, st) != cudaSuccess)
         return SC_ERR_CUDA;

@@ -26,18 +26,19 @@ def sc(binding):
     s.close()
 
 
-def _run(sc, binding, A, W, L, Lmax, scale_a, scale_w, seed, stream_id=0, group=1, want_P=True, quant=0):
+def _run(sc, binding, A, W, L, Lmax, scale_a, scale_w, seed, stream_id=0, group=1, want_P=True, quant=0, core=0):
     import torch
     params = binding.make_params(mode=0, scale_a=scale_a, scale_w=scale_w, group=group, seed=seed, stream_id=stream_id,
-                                 quant=quant)
+                                 quant=quant, core=core)
     dL = None if L is None else torch.from_numpy(np.ascontiguousarray(L, dtype=np.int32)).cuda()
     P, C = sc.matmul_cbsg(torch.from_numpy(A).cuda(), torch.from_numpy(W).cuda(), dL, Lmax, params, want_P)
     torch.cuda.synchronize()
     return (None if P is None else P.cpu().numpy()), C.cpu().numpy()
 
 
+@pytest.mark.parametrize("core", [4, 5])
 @pytest.mark.parametrize("seed,scale_w", [(3, PER_TENSOR), (4, PER_ROW)])
-def test_small_ragged_full(sc, binding, oracle, seed, scale_w):
+def test_small_ragged_full(sc, binding, oracle, seed, scale_w, core):
     """Several row tiles, a padded column tile, a depth tail; per-row lengths over the whole range 0..256."""
     rng = np.random.default_rng(seed)
     M, K, N = 203, 70, 150
@@ -45,7 +46,7 @@ def test_small_ragged_full(sc, binding, oracle, seed, scale_w):
     W = (0.02 * rng.standard_normal((K, N))).astype(np.float32)
     L = rng.integers(0, 257, size=M).astype(np.int32)
     L[:4] = [0, 256, 1, 255]
-    P, C = _run(sc, binding, A, W, L, 256, PER_ROW, scale_w, seed, stream_id=2)
+    P, C = _run(sc, binding, A, W, L, 256, PER_ROW, scale_w, seed, stream_id=2, core=core)
     ref = oracle.matmul_cbsg(A, W, L, PER_ROW, scale_w, seed=seed, stream_id=2)
     assert np.array_equal(P, ref["P"])
     assert T.close_enough(C, ref["C"])
@@ -84,12 +85,13 @@ def test_groups_uniform_and_exact_full_length(sc, binding, oracle):
     assert P2 is None and T.close_enough(C2, ref2["C"])
 
 
-def test_vit_b_fc1_sampled(sc, binding, oracle):
+@pytest.mark.parametrize("core", [0, 5])
+def test_vit_b_fc1_sampled(sc, binding, oracle, core):
     """Config-2 shape (1576 x 768 x 3072) at L = 128: sampled rows x columns against the oracle."""
     w = wl.VIT_B_FC1
     A, W = wl.make_inputs(w)
     L = np.full(w.M, 128, dtype=np.int32)
-    P, C = _run(sc, binding, A, W, L, 128, PER_ROW, PER_TENSOR, w.seed)
+    P, C = _run(sc, binding, A, W, L, 128, PER_ROW, PER_TENSOR, w.seed, core=core)
     rows, cols = wl.sample_rows_cols(w, L, 10, 24)
     ref = oracle.matmul_cbsg(A, W, L, PER_ROW, PER_TENSOR, seed=w.seed, row_sel=rows, col_sel=cols)
     assert np.array_equal(P[np.ix_(rows, cols)], ref["P"])
