@@ -120,36 +120,54 @@ struct UmmaDev {
 
 struct UItem {
     int32_t rt, ct, q0, q1, n_raw;
+    int32_t adv;            // how far the walk moves on (the piece's units plus any hand-over charge walked over)
 };
 
 // Work decomposition: the plan lists, per row tile, the running total of stage units (one unit = one TMA stage of
 // kStagePlanes planes of one (row tile, column tile)).  CTA c owns the contiguous run [c T / G, (c + 1) T / G) of the
-// T units, cutting tiles where its run begins and ends: all CTAs get the same amount of MMA work whatever the tile
+// T units, cutting tiles where its run begins and ends: all CTAs get the same amount of work whatever the tile
 // count is, and the pieces of a cut tile meet in the global accumulators.  Every role of a CTA walks the same pieces.
+// A piece boundary (accumulator hand-over, pipeline refill) costs about as much as a few units, so the plan charges every
+// (row tile, column tile) `charge` virtual units in front of its real ones (PlanHeader.pad[1]): CTAs whose runs cross
+// many short tiles receive fewer real units, and all CTAs finish together when lengths are ragged.
 __device__ __forceinline__ int32_t u_run_begin(const PlanHeader &plan, int32_t cta)
 {
     return (int32_t)((long long)plan.total_items * cta / (long long)gridDim.x);
 }
 
+// The next piece with work at or after position `pos` of the run ending at `end` (n_raw == 0: none is left).
 __device__ __forceinline__ UItem u_piece(const PlanHeader &plan, const int32_t *prefix, const int32_t *tile_planes,
                                          int32_t pos, int32_t end)
 {
-    int32_t lo = 0, hi = plan.n_row_tiles;               // largest row tile with prefix <= pos (skips empty tiles)
-    while (hi - lo > 1) {
-        const int32_t mid = (lo + hi) >> 1;
-        if (__ldg(prefix + mid) <= pos) lo = mid; else hi = mid;
-    }
+    const int32_t charge = plan.pad[1];
     UItem it;
-    it.rt = lo;
-    const int32_t planes = __ldg(tile_planes + lo);
-    const int32_t stages = (planes + kStagePlanes - 1) / kStagePlanes;
-    const int32_t local = pos - __ldg(prefix + lo);
-    it.ct = local / stages;
-    const int32_t s0 = local - it.ct * stages;
-    const int32_t s1 = min(stages, s0 + (end - pos));
-    it.q0 = s0 * kStagePlanes;
-    it.q1 = min(s1 * kStagePlanes, planes);
-    it.n_raw = s1 - s0;
+    it.n_raw = 0;
+    it.adv = 0;
+    while (pos < end) {
+        int32_t lo = 0, hi = plan.n_row_tiles;           // largest row tile with prefix <= pos (skips empty tiles)
+        while (hi - lo > 1) {
+            const int32_t mid = (lo + hi) >> 1;
+            if (__ldg(prefix + mid) <= pos) lo = mid; else hi = mid;
+        }
+        const int32_t planes = __ldg(tile_planes + lo);
+        const int32_t stages = (planes + kStagePlanes - 1) / kStagePlanes;
+        const int32_t charged = stages + charge;         // positions of one column tile: the charge, then the real units
+        const int32_t local = pos - __ldg(prefix + lo);
+        const int32_t ct = local / charged;
+        const int32_t x0 = local - ct * charged;
+        const int32_t x1 = min(charged, x0 + (end - pos));
+        const int32_t s0 = max(x0 - charge, 0), s1 = max(x1 - charge, 0);
+        it.adv += x1 - x0;
+        pos += x1 - x0;
+        if (s1 > s0) {
+            it.rt = lo;
+            it.ct = ct;
+            it.q0 = s0 * kStagePlanes;
+            it.q1 = min(s1 * kStagePlanes, planes);
+            it.n_raw = s1 - s0;
+            return it;
+        }
+    }
     return it;
 }
 
@@ -210,7 +228,7 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
             n += __shfl_xor_sync(0xFFFFFFFFu, n, o);
             shortest = min(shortest, __shfl_xor_sync(0xFFFFFFFFu, shortest, o));
         }
-        const int32_t mean = plan.total_items / (n * plan.n_col_tiles + (int32_t)gridDim.x);
+        const int32_t mean = (plan.total_items - plan.pad[1] * n * plan.n_col_tiles) / (n * plan.n_col_tiles + (int32_t)gridDim.x);
         if (lane == 0) *s_single = min(mean, shortest) >= kSingleAccUnits ? 1 : 0;
     }
     u_fence_before();
@@ -254,7 +272,8 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
             bool ok = true;
             for (int32_t pos = u_run_begin(plan, blockIdx.x), end = u_run_begin(plan, blockIdx.x + 1); pos < end && ok && !*s_abort;) {
                 const UItem it = u_piece(plan, prefix, tile_planes, pos, end);
-                pos += it.n_raw;
+                pos += it.adv;
+                if (it.n_raw == 0) break;
                 // one box holds kRawUnits units; the last box of a piece may reach past it (those planes are not used)
                 for (int32_t k = 0; k < (it.n_raw + kRawUnits - 1) / kRawUnits; ++k, ++raw_cnt) {
                     const uint32_t s = raw_cnt % kRawStages;
@@ -290,7 +309,8 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
             constexpr uint32_t kStepDesc = (2u * kLboB) >> 4, kStageDesc = kOpStageBytes >> 4;
             for (int32_t pos = u_run_begin(plan, blockIdx.x), end = u_run_begin(plan, blockIdx.x + 1); pos < end && ok && !*s_abort;) {
                 const UItem it = u_piece(plan, prefix, tile_planes, pos, end);
-                pos += it.n_raw;
+                pos += it.adv;
+                if (it.n_raw == 0) break;
                 const uint32_t b = single ? 0u : acc_cnt & 1u, acc_phase = (single ? acc_cnt : acc_cnt >> 1) & 1u;
                 const uint32_t first = op_cnt % kIssuers;        // owner of the item's first stage: it overwrites
                 site = 2;
@@ -339,7 +359,8 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
         uint32_t acc_cnt = 0, chunk_cnt = 0;
         for (int32_t pos = u_run_begin(plan, blockIdx.x), end = u_run_begin(plan, blockIdx.x + 1); pos < end && !*s_abort;) {
             const UItem it = u_piece(plan, prefix, tile_planes, pos, end);
-            pos += it.n_raw;
+            pos += it.adv;
+                if (it.n_raw == 0) break;
             const int64_t r = (int64_t)it.rt * kTileM + quarter * 32 + lane;
             int32_t src = __ldg(p.perm + r);
             // nothing of this row in the chunk: its stream ends at or before the first position block of the chunk
@@ -406,7 +427,7 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
         constexpr int kStagePl = kStagePp;            // A plane words of one operand stage held in registers
         constexpr int kSignWords = a_signed ? 4 : 1;
         struct AIter {
-            int32_t pos, end, j, n_ops, my_len, rt, q0, q1, n_raw;
+            int32_t pos, end, j, n_ops, my_len, rt, q0, q1, n_raw, adv;
             uint32_t op;
             bool valid;
         };
@@ -414,6 +435,8 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
             x.valid = x.pos < x.end;
             if (!x.valid) return;
             const UItem it = u_piece(plan, prefix, tile_planes, x.pos, x.end);
+            x.adv = it.adv;
+            if (it.n_raw == 0) { x.valid = false; return; }
             x.rt = it.rt; x.q0 = it.q0; x.q1 = it.q1; x.n_raw = it.n_raw;
             x.n_ops = it.n_raw * kOpsPerRaw;
             x.j = 0;
@@ -422,7 +445,7 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
         auto advance = [&](AIter &x, int n) {
             for (int a = 0; a < n && x.valid; ++a) {
                 ++x.op;
-                if (++x.j == x.n_ops) { x.pos += x.n_raw; load_piece(x); }
+                if (++x.j == x.n_ops) { x.pos += x.adv; load_piece(x); }
             }
         };
         auto fetch = [&](const AIter &x, uint32_t (&dst)[kStagePl], uint32_t (&sgn)[kSignWords]) {
@@ -512,7 +535,8 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
         bool ok = true;
         for (int32_t pos = u_run_begin(plan, blockIdx.x), end = u_run_begin(plan, blockIdx.x + 1); pos < end && ok && !*s_abort;) {
             const UItem it = u_piece(plan, prefix, tile_planes, pos, end);
-            pos += it.n_raw;
+            pos += it.adv;
+                if (it.n_raw == 0) break;
             for (int32_t k = 0; k < (it.n_raw + kRawUnits - 1) / kRawUnits && ok; ++k, ++raw_cnt) {
                 const uint32_t s = raw_cnt % kRawStages;
                 const int ops_here = min(kRawUnits, it.n_raw - k * kRawUnits) * kOpsPerRaw;    // units present in this box

@@ -15,6 +15,10 @@ constexpr int kPlanThreads = 1024;
 // call (256 x 256 tiles on pairs of SMs; an odd row tile or a ragged last column tile is padding) costs no more MMA time
 // than the one-SM core's (128 x 192 tiles) after its measured advantage per multiply-accumulate on long pieces (7 %).
 constexpr int32_t kPairMinUnits = 96;
+// One-SM tensor-core core: a piece boundary costs about this many stage units (accumulator hand-over, pipeline refill); the
+// prefix sums charge it to every (row tile, column tile) so that equal runs are runs of equal time (see u_piece).
+constexpr int32_t kPieceChargeUnits = 4;      // measured: 0 / 4 / 8 / 12 units give 0.120 / 0.117 / 0.117 / 0.121 ms on the per-row mixed
+                                              // ViT-B/16 qkv configuration and 2.03 / 1.94 / 1.96 / 1.99 ms on the grouped DiT-like one
 constexpr long long kPairAdvantagePct = 107;
 
 struct PairChoice {
@@ -82,12 +86,15 @@ __device__ void finish_plan(int32_t n_row_tiles, int32_t n_col_tiles, int32_t ta
     }
     __syncthreads();
     const int32_t chunk = *s_chunk;
+    const int32_t charge = wave_ctas > 0 ? kPieceChargeUnits : 0;
 
     // exclusive prefix sums of the items per tile: every thread owns a run of consecutive tiles
     const int32_t per = (n_row_tiles + kPlanThreads - 1) / kPlanThreads;
     const int32_t t0 = min(tid * per, n_row_tiles), t1 = min(t0 + per, n_row_tiles);
     int32_t local = 0;
-    for (int32_t rt = t0; rt < t1; ++rt) local += (tile_planes[rt] + chunk - 1) / chunk * n_col_tiles;
+    // items of one row tile: per column tile its chunks, plus (tensor-core core) the charge for the piece boundary
+    auto tile_items = [&](int32_t planes) { return planes > 0 ? ((planes + chunk - 1) / chunk + charge) * n_col_tiles : 0; };
+    for (int32_t rt = t0; rt < t1; ++rt) local += tile_items(tile_planes[rt]);
     int32_t incl = local;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -110,7 +117,7 @@ __device__ void finish_plan(int32_t n_row_tiles, int32_t n_col_tiles, int32_t ta
     int32_t run = s_scan[warp] + incl - local;
     for (int32_t rt = t0; rt < t1; ++rt) {
         prefix[rt] = run;
-        run += (tile_planes[rt] + chunk - 1) / chunk * n_col_tiles;
+        run += tile_items(tile_planes[rt]);
     }
     if (tid == kPlanThreads - 1) {
         prefix[n_row_tiles] = run;
@@ -130,6 +137,7 @@ __device__ void finish_plan(int32_t n_row_tiles, int32_t n_col_tiles, int32_t ta
                                        t_pair * 100 <= t_single * kPairAdvantagePct)) ? 1 : 0;
         }
         plan->pad[0] = use_pair;                      // which tensor-core core runs: 1 = the two-SM core
+        plan->pad[1] = charge;                        // virtual units in front of every (row tile, column tile) in the prefix sums
         scratch[kSlotTicket] = 0;
         scratch[kSlotAnyNegA] = 0;                    // the encode of A sets it again if it meets a negative element
         scratch[kSlotLmaxActual] = longest / planes_per_len;
