@@ -36,7 +36,8 @@ L2_FLUSH_BYTES = 256 << 20
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one core-kernel launch, from an
 # `ncu --set full` capture of this command on the workload named by the key.
-NCU_CORE_TRAFFIC_BYTES = {("vit_b16_fc1", "alu"): 85.4e6, ("vit_b16_fc1", "umma"): 90.3e6}
+NCU_CORE_TRAFFIC_BYTES = {("vit_b16_fc1", "alu"): 85.4e6, ("vit_b16_fc1", "umma"): 93.8e6,
+                          ("vit_l14_fc1_L128", "umma"): 5.35e9}
 
 FP4_TO_BF16_NOMINAL = 4.0       # dense tensor peaks: 9 PFLOP/s fp4 vs 2.25 PFLOP/s bf16
 

@@ -112,13 +112,15 @@ static bool choose_pair(sc_ctx_impl *c, const sc_params *params, bool umma, int6
     if (pair_core_clusters(params->mode, c->sm_count, &out->clusters) != cudaSuccess) return false;
     if (out->clusters < 1) out->mode = 0;
     if (out->mode == 1) {
-        // The plan selects the two-SM core only if its tiling costs at most 7 % more MMA time than the one-SM core's (its
-        // measured advantage on long pieces).  Where the shape alone already rules that out (an odd row tile, a ragged last
-        // column tile: ragged lengths only add to it), the two-SM kernel is not enqueued at all.
+        // The plan selects the two-SM core only if its tiling costs at most 10 % more MMA time than the one-SM core's (its
+        // measured advantage on long pieces; shorter pieces tighten the condition).  Where the shape alone already rules
+        // that out (an odd row tile, a ragged last column tile: ragged lengths only add to it), the two-SM kernel is not
+        // enqueued at all.
         const int64_t row_tiles = m_pad / kTileM, pairs = (row_tiles + 1) / 2;
         const int64_t t_pair = pairs * out->col_tiles * pair_core_tile_cols() * 2;
-        const int64_t t_single = row_tiles * ((N + kTileNUmma - 1) / kTileNUmma) * kTileNUmma;
-        if (t_pair * 100 > t_single * 107) out->mode = 0;
+        const int64_t tile_n = umma_tile_cols(N);
+        const int64_t t_single = row_tiles * ((N + tile_n - 1) / tile_n) * tile_n;
+        if (t_pair * 100 > t_single * 110) out->mode = 0;
     }
     return true;
 }
@@ -395,7 +397,8 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     // not wait for it.  With phase timing on, everything stays on the caller's stream in the order of the phases.
     const bool fork = !pw && c->overlap && !c->profiling;
     cudaStream_t sw = fork ? c->side : st;          // the stream of the W-side work
-    const int64_t n_col_tiles = umma ? (N + kTileNUmma - 1) / kTileNUmma : (N + kTileN - 1) / kTileN;
+    const int32_t tile_n = umma_tile_cols(N);                        // column tile of the one-SM tensor-core core
+    const int64_t n_col_tiles = umma ? (N + tile_n - 1) / tile_n : (N + kTileN - 1) / kTileN;
     // a1: scales (the per-row scale of A is also the row metric of Sec. 4.4)
     auto scales = [&]() -> bool {
         if (!fork && compute_scales(c, A, M, K, 0, params->scale_a, sigma_a, st, B) != cudaSuccess) return false;
@@ -408,7 +411,7 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     auto plan_rows = [&]() -> bool {
         if (launch_plan(L, M, params->group, Lmax, w.kw, ppq, m_pad_b, n_col_tiles, umma ? 0 : c->sm_count * 16,
                         umma ? c->sm_count : 0, l_rows, perm, l_sorted, plan, c->scratch, st, B, pos_block, pair_col_tiles,
-                        pair_mode ? pair_clusters : 0, pair_mode == 2) != cudaSuccess)
+                        pair_mode ? pair_clusters : 0, pair_mode == 2, tile_n) != cudaSuccess)
             return false;
         // the W encode stops at the longest length of the call
         if (fork && (cudaEventRecord(c->ev_plan, st) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_plan, 0) != cudaSuccess))
@@ -463,6 +466,7 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     ca.a_planes = w.a_planes / ppq_alloc * ppq;                          // planes the operands really have
     ca.w_planes = w.w_planes / ppq_alloc * ppq;
     ca.w_sign = signs ? w_sign : nullptr; ca.a_sign = signs ? a_sign : nullptr; ca.pos_block = pos_block;
+    ca.tile_n = tile_n;
     ca.M = Mt; ca.N = N; ca.mode = params->mode;
     ca.tiles_m = (int32_t)(m_pad_b / kTileM); ca.w_batch_cols = n_pad_b;
     ca.variant = variant;
@@ -570,12 +574,13 @@ sc_status sc_matmul_cbsg(sc_ctx *ctx, const float *A, const float *W, int64_t M,
     mark(1);
     if (launch_cbsg_setup(params->seed, params->stream_id, tables, L, n_groups, Lmax, l_core, status, st) != cudaSuccess)
         return SC_ERR_CUDA;
-    const int64_t n_col_tiles = (N + kTileNUmma - 1) / kTileNUmma;
+    const int32_t tile_n = umma_tile_cols(N);
+    const int64_t n_col_tiles = (N + tile_n - 1) / tile_n;
     PairLaunch pair;
     if (!choose_pair(c, params, true, w.m_pad, N, 1, &pair)) return SC_ERR_CUDA;
     if (launch_plan(l_core, M, params->group, core_lmax, w.kw, 1, w.m_pad, n_col_tiles, 0, c->sm_count, l_rows,
                     perm, l_sorted, plan, c->scratch, st, 1, 1, pair.col_tiles, pair.mode ? pair.clusters : 0,
-                    pair.mode == 2) != cudaSuccess)
+                    pair.mode == 2, tile_n) != cudaSuccess)
         return SC_ERR_CUDA;
     if (cudaMemsetAsync(acc, 0, sizeof(int32_t) * (size_t)M * (size_t)N, st) != cudaSuccess) return SC_ERR_CUDA;
     mark(2);
@@ -595,6 +600,7 @@ sc_status sc_matmul_cbsg(sc_ctx *ctx, const float *A, const float *W, int64_t M,
     ca.perm = perm; ca.l_sorted = l_sorted; ca.plan = plan; ca.kw = (int32_t)w.kw; ca.ppq = 1;
     ca.acc = acc; ca.scratch = c->scratch; ca.sm_count = c->sm_count; ca.Lmax = core_lmax;
     ca.pop_a = nullptr; ca.pop_w = nullptr;
+    ca.tile_n = tile_n;
     if (launch_core_umma(ca, st) != cudaSuccess) return SC_ERR_CUDA;
     if (pair.mode && launch_core_umma_pair(ca, pair.clusters, pair.mode == 2, st) != cudaSuccess) return SC_ERR_CUDA;
     mark(5);

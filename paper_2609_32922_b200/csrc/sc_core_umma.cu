@@ -113,6 +113,9 @@ struct UmmaDev {
     const uint32_t *w_sign;           // unipolar: [depth word][n_pad][4] nibble sign words of W ...
     const uint32_t *a_sign;           // ... and [depth word][m_pad][4] of A
     int64_t n_pad;                    // padded W stream rows in all
+    int32_t tile_n;                   // output columns per tile: a multiple of 32, at most kUN (the shared-memory layout, the
+                                      // TMA box and the accumulator are kUN wide; columns from tile_n on are not expanded,
+                                      // not multiplied and not read back)
 };
 
 // (The bit -> 4-bit float expansions u_expand_bits / u_expand_signed_a / u_expand_signed_w live in sc_device.cuh,
@@ -171,10 +174,13 @@ __device__ __forceinline__ UItem u_piece(const PlanHeader &plan, const int32_t *
     return it;
 }
 
-template <int kMode>
+// kNarrow: the tile is narrower than kUN columns (UmmaDev.tile_n, narrow products); otherwise the width is the constant
+// kUN and every test against it folds away (the kernel is sensitive to each instruction on its expander paths).
+template <int kMode, bool kNarrow>
 __global__ void __launch_bounds__(kUThreads, 1)
 core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
 {
+    const int32_t tile_n = kNarrow ? p.tile_n : kUN;
     // An MMA K-step of 64 elements is two (depth word, position) pairs = two planes of either operand.
     constexpr int kPpq = 2;
     constexpr int kStepsPerRaw = kStagePlanes / kPpq;              // MMA steps in one raw stage
@@ -281,7 +287,7 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
                     if (!ok) break;
                     u_mbar_expect_tx(bar(kRawFull + s), kRawStageBytes);
                     const uint32_t dst = raw_addr + s * kRawStageBytes;
-                    u_tma_load_2d(dst, &map_w, (int32_t)((it.rt / p.tiles_m) * p.w_batch_cols) + it.ct * kUN,
+                    u_tma_load_2d(dst, &map_w, (int32_t)((it.rt / p.tiles_m) * p.w_batch_cols) + it.ct * tile_n,
                                   it.q0 + k * kRawPlanes, bar(kRawFull + s));
                 }
             }
@@ -307,6 +313,7 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
             int site = 0;
             const uint64_t desc0 = u_smem_desc(ops_addr, kLboB);
             constexpr uint32_t kStepDesc = (2u * kLboB) >> 4, kStageDesc = kOpStageBytes >> 4;
+            const uint32_t idesc = u_idesc_fp4(kTileM, (uint32_t)tile_n);
             for (int32_t pos = u_run_begin(plan, blockIdx.x), end = u_run_begin(plan, blockIdx.x + 1); pos < end && ok && !*s_abort;) {
                 const UItem it = u_piece(plan, prefix, tile_planes, pos, end);
                 pos += it.adv;
@@ -331,7 +338,7 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
                     const uint32_t a_base = tmem_base + a_ring_col + a_slot(op_cnt) * (kOpSteps * 8u);
 #pragma unroll
                     for (int st = 0; st < kOpSteps; ++st) {
-                        u_mma_fp4_ts(d_tmem, a_base + st * 8u, bdesc + (uint64_t)(st * kStepDesc), u_idesc_fp4(kTileM, kUN),
+                        u_mma_fp4_ts(d_tmem, a_base + st * 8u, bdesc + (uint64_t)(st * kStepDesc), idesc,
                                      (uint32_t)((j | st) != 0), tmem_base + kSfCol, tmem_base + kSfCol + 16u);
                         if (j == 0 && st == 0) u_mbar_arrive(bar(kAccStarted + b));     // the overwrite is in the pipe
                     }
@@ -369,7 +376,7 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
             if (!u_mbar_wait_warp(bar(kAccFull + b), acc_phase, s_abort, lane)) { if (lane == 0) give_up(5, acc_cnt, 0); break; }
             u_fence_after();
 #pragma unroll 1
-            for (int c = 0; c < kUN / 32; ++c, ++chunk_cnt) {
+            for (int c = 0; c * 32 < tile_n; ++c, ++chunk_cnt) {
                 uint32_t v[32];
                 u_tmem_ld32(tmem_base + b * kAccCols + (uint32_t)c * 32u + ((quarter * 32u) << 16), v);
                 // the accumulators hold exact fp32 integers
@@ -378,16 +385,18 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
                 uint32_t *buf = tile0 + (chunk_cnt & 1u) * (32 * kEpiStride);
                 // the bulk operation that read this buffer two chunks ago has finished reading
                 asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                const int64_t col0 = (int64_t)it.ct * kUN + c * 32;
-                if (bulk_ok && col0 + 32 <= p.N) {
+                const int64_t col0 = (int64_t)it.ct * tile_n + c * 32;
+                // columns of this chunk that exist: inside the tile and inside the matrix
+                const int32_t width = (int32_t)min((int64_t)min(32, tile_n - c * 32), p.N - col0);
+                if (bulk_ok && width > 0 && (width & 3) == 0) {
                     uint4 *dst = reinterpret_cast<uint4 *>(buf + lane * kEpiStride);
 #pragma unroll
                     for (int j = 0; j < 8; ++j) dst[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     if (src >= 0)
-                        asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.s32 [%0], [%1], 128;"
-                                     ::"l"(p.acc + (int64_t)src * p.N + col0), "r"(u_smem(dst)) : "memory");
-                } else {
+                        asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.s32 [%0], [%1], %2;"
+                                     ::"l"(p.acc + (int64_t)src * p.N + col0), "r"(u_smem(dst)), "r"((uint32_t)width * 4u) : "memory");
+                } else if (width > 0) {
                     __syncwarp();
 #pragma unroll
                     for (int k = 0; k < 32; ++k) buf[lane * kEpiStride + k] = v[k];
@@ -397,7 +406,7 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
                     for (int rr = 0; rr < 32; ++rr) {
                         const int32_t s_rr = __shfl_sync(0xFFFFFFFFu, src, rr);
                         const uint32_t val = buf[rr * kEpiStride + lane];
-                        if (s_rr >= 0 && col < p.N && val != 0u) atomicAdd(p.acc + (int64_t)s_rr * p.N + col, (int32_t)val);
+                        if (s_rr >= 0 && lane < width && val != 0u) atomicAdd(p.acc + (int64_t)s_rr * p.N + col, (int32_t)val);
                     }
                     __syncwarp();
                 }
@@ -548,7 +557,7 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
                 if (kMode == SC_UNIPOLAR_AND) {
                     const int first_own = (group + kWGroups - (int)(op_cnt % kWGroups)) % kWGroups;
                     const uint4 *sign_col = reinterpret_cast<const uint4 *>(p.w_sign) + (int64_t)(it.rt / p.tiles_m) * p.w_batch_cols +
-                                            (int64_t)it.ct * kUN + row;
+                                            (int64_t)it.ct * tile_n + row;
 #pragma unroll
                     for (int o = 0; o < kOwnMax; ++o) {
                         const int i = first_own + o * kWGroups;
@@ -556,7 +565,8 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
                         const int32_t wd = pp0 % (kPosBlockSigned * p.planes_per_len) / kPosBlockSigned;
 #pragma unroll
                         for (int c = 0; c < kWCols; ++c)
-                            sg_box[o][c] = i < ops_here ? __ldg(sign_col + (int64_t)wd * p.n_pad + c * (kUN / kWCols)) : make_uint4(0u, 0u, 0u, 0u);
+                            sg_box[o][c] = (i < ops_here && row + c * (kUN / kWCols) < tile_n)
+                                               ? __ldg(sign_col + (int64_t)wd * p.n_pad + c * (kUN / kWCols)) : make_uint4(0u, 0u, 0u, 0u);
                     }
                 }
                 int own = 0;
@@ -576,6 +586,7 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
 #pragma unroll
                     for (int c = 0; c < kWCols; ++c) {
                         const int idx = row + c * (kUN / kWCols);
+                        if (idx >= tile_n) continue;               // beyond the tile: nothing to expand
 #pragma unroll
                         for (int q = 0; q < kStagePl; ++q) pl[c][q] = raw_w[(i * kStagePl + q) * kUN + idx];
                         if (kMode == SC_UNIPOLAR_AND) sg[c] = own == 0 ? sg_box[0][c] : sg_box[kOwnMax - 1][c];
@@ -591,6 +602,7 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
                     if (!ok) break;
 #pragma unroll
                     for (int c = 0; c < kWCols; ++c) {
+                        if (row + c * (kUN / kWCols) >= tile_n) continue;
                         uint8_t *op_b = ops + (size_t)t * kOpStageBytes + (row + c * (kUN / kWCols)) * 16;
                         uint32_t sn[4] = {0u, 0u, 0u, 0u};
                         if (kMode == SC_UNIPOLAR_AND) { sn[0] = sg[c].x; sn[1] = sg[c].y; sn[2] = sg[c].z; sn[3] = sg[c].w; }
@@ -771,18 +783,18 @@ cudaError_t launch_col_corrections(const uint32_t *w_streams, int64_t n_pad, int
 bool make_plane_map(CUtensorMap *map, const uint32_t *base, int64_t row_words, int64_t planes, int box_words,
                     int box_planes);
 
-template <int kMode>
+template <int kMode, bool kNarrow>
 static cudaError_t launch_umma_mode(const CUtensorMap &mw, const UmmaDev &dev, int sm_count,
                                     cudaStream_t st)
 {
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(core_umma_kernel<kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(core_umma_kernel<kMode, kNarrow>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kUmmaSmem);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    core_umma_kernel<kMode><<<sm_count, kUThreads, kUmmaSmem, st>>>(mw, dev);
+    core_umma_kernel<kMode, kNarrow><<<sm_count, kUThreads, kUmmaSmem, st>>>(mw, dev);
     count_launches(1);
     return cudaGetLastError();
 }
@@ -796,11 +808,17 @@ cudaError_t launch_core_umma(const CoreArgs &a, cudaStream_t st)
     dev.perm = a.perm; dev.l_sorted = a.l_sorted; dev.plan = a.plan; dev.acc = a.acc; dev.scratch = a.scratch;
     dev.N = a.N; dev.planes_per_len = a.kw; dev.pos_block = a.pos_block;
     dev.w_sign = a.w_sign; dev.a_sign = a.a_sign; dev.n_pad = a.n_pad;
+    dev.tile_n = a.tile_n;
+    if (a.tile_n < 32 || a.tile_n > kUN || a.tile_n % 32 != 0) return cudaErrorInvalidValue;
     if (a.mode == SC_UNIPOLAR_AND && (a.pos_block != kPosBlockSigned || !a.w_sign || !a.a_sign)) return cudaErrorInvalidValue;
     if (a.mode != SC_UNIPOLAR_AND && a.pos_block != 1) return cudaErrorInvalidValue;
     dev.tiles_m = a.tiles_m; dev.w_batch_cols = a.w_batch_cols;
-    if (a.mode == SC_UNIPOLAR_AND) return launch_umma_mode<SC_UNIPOLAR_AND>(mw, dev, a.sm_count, st);
-    return launch_umma_mode<SC_BIPOLAR_XNOR>(mw, dev, a.sm_count, st);
+    const bool narrow = a.tile_n != kUN;
+    if (a.mode == SC_UNIPOLAR_AND)
+        return narrow ? launch_umma_mode<SC_UNIPOLAR_AND, true>(mw, dev, a.sm_count, st)
+                      : launch_umma_mode<SC_UNIPOLAR_AND, false>(mw, dev, a.sm_count, st);
+    return narrow ? launch_umma_mode<SC_BIPOLAR_XNOR, true>(mw, dev, a.sm_count, st)
+                  : launch_umma_mode<SC_BIPOLAR_XNOR, false>(mw, dev, a.sm_count, st);
 }
 
 }  // namespace sc

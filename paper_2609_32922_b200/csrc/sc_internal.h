@@ -14,6 +14,16 @@ constexpr int kTileM = 128;          // rows of A per CTA tile (sorted order)
 constexpr int kTileN = 128;          // output columns per CTA tile (ALU cores)
 constexpr int kTileNUmma = 192;      // output columns per CTA tile (tensor-core core)
 constexpr int kColPad = 384;         // W stream rows are padded to a multiple of both tile widths
+// Column tile of the one-SM tensor-core core for N output columns: the columns are spread evenly over the tiles a width of
+// kTileNUmma needs, in multiples of 32 (tiles then start on 128-byte boundaries of the plane rows; with multiples of 16 --
+// N = 1024 as six tiles of 176 -- the weight boxes straddle one more line each and the core ran 6 - 19 % slower than with
+// 192), so that narrow products cost less (N = 64: one tile of 64; N = 257: two of 160 instead of 192).
+inline int umma_tile_cols(int64_t N)
+{
+    const int64_t tiles = (N + kTileNUmma - 1) / kTileNUmma;
+    const int64_t w = ((N + tiles - 1) / tiles + 31) / 32 * 32;
+    return (int)(w < kTileNUmma ? w : kTileNUmma);
+}
 constexpr int kStagePlanes = 16;     // stream planes per pipeline stage
 constexpr int kStages = 4;           // TMA pipeline depth
 constexpr int kScratchBytes = 64 * 1024;
@@ -137,7 +147,7 @@ cudaError_t launch_plan(const int32_t *L, int64_t M, int32_t group, int32_t Lmax
                         int64_t m_pad, int64_t n_col_tiles, int32_t target_items, int32_t wave_ctas,
                         int32_t *l_rows, int32_t *perm, int32_t *l_sorted, PlanHeader *plan, int32_t *scratch,
                         cudaStream_t st, int64_t batch = 1, int32_t pos_block = 1, int32_t pair_col_tiles = 0,
-                        int32_t pair_clusters = 0, int32_t pair_force = 0);
+                        int32_t pair_clusters = 0, int32_t pair_force = 0, int32_t single_tile_cols = kTileNUmma);
 
 struct EncodeArgs {
     const float *X;
@@ -187,6 +197,7 @@ struct CoreArgs {
     const uint32_t *w_sign = nullptr;   // unipolar tensor-core core: [kw][n_pad][4] nibble sign words of W ...
     const uint32_t *a_sign = nullptr;   // ... and [kw][m_pad][4] of A (sorted row order)
     int32_t pos_block = 1;       // block size of the stream positions in both operands' planes
+    int32_t tile_n = kTileNUmma; // one-SM tensor-core core: output columns per tile (umma_tile_cols)
     int32_t *pop_a;              // [M] ones of each row of A below its own end (tensor-core core, bipolar)
     const int32_t *pop_w;        // [(Lmax + 1) x n_pad] prefix ones of each W column (tensor-core core, bipolar)
 };

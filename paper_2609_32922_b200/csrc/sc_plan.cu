@@ -9,22 +9,25 @@ namespace sc {
 
 constexpr int kPlanThreads = 1024;
 
-// The work list over all row tiles (run by one CTA of kPlanThreads threads): chunk size, item prefix sums, totals.
-// Two-SM core (sc_core_umma2.cu): it has one accumulator, so a piece boundary drains its pipeline; it is selected when
-// the pieces are long -- min(mean stage units per piece, shortest tile pair) at least kPairMinUnits -- and its tiling of the
-// call (256 x 256 tiles on pairs of SMs; an odd row tile or a ragged last column tile is padding) costs no more MMA time
-// than the one-SM core's (128 x 192 tiles) after its measured advantage per multiply-accumulate on long pieces (7 %).
-constexpr int32_t kPairMinUnits = 96;
+// Two-SM core (sc_core_umma2.cu): it has one accumulator, so a piece boundary drains its pipeline (about kPairDrainUnits stage
+// units, against the kPieceChargeUnits of the one-SM core), it works on pairs of row tiles and on 256-column tiles (an odd row
+// tile or a ragged last column tile is padding), and on long pieces it needs 10 % less time per multiply-accumulate.  It is
+// selected when its estimated time is the shorter one:
+//     t_pair (u + kPairDrainUnits) <= 1.10 t_single (u + kPieceChargeUnits),   u = min(mean units per piece, shortest tile pair),
+// t = stage units x column tiles x tile columns / SMs per tile (MMA time up to a common factor).  Measured against the forced
+// choices on the ViT-L/14 sweep and the ragged configurations (profiles/core_umma_pair_kernel_*.md).
+constexpr long long kPairDrainUnits = 14;
+constexpr long long kPairAdvantagePct = 110;
 // One-SM tensor-core core: a piece boundary costs about this many stage units (accumulator hand-over, pipeline refill); the
 // prefix sums charge it to every (row tile, column tile) so that equal runs are runs of equal time (see u_piece).
 constexpr int32_t kPieceChargeUnits = 4;      // measured: 0 / 4 / 8 / 12 units give 0.120 / 0.117 / 0.117 / 0.121 ms on the per-row mixed
                                               // ViT-B/16 qkv configuration and 2.03 / 1.94 / 1.96 / 1.99 ms on the grouped DiT-like one
-constexpr long long kPairAdvantagePct = 107;
 
 struct PairChoice {
     int32_t col_tiles;      // column tiles of the two-SM core (0: that core is not available for the call)
     int32_t clusters;       // CTA pairs it runs with
     int32_t force;          // select it whatever the lengths are
+    int32_t single_cols;    // columns per tile of the one-SM core (its n_col_tiles tiles are compared with)
 };
 
 __device__ void finish_plan(int32_t n_row_tiles, int32_t n_col_tiles, int32_t target_items, int32_t wave_ctas,
@@ -132,9 +135,9 @@ __device__ void finish_plan(int32_t n_row_tiles, int32_t n_col_tiles, int32_t ta
             const long long mean = (long long)s_cost[1] * pair.col_tiles / pieces;
             // MMA time of the two tilings, up to a common factor: units x column tiles x tile columns / SMs per tile
             const long long t_pair = (long long)s_cost[1] * pair.col_tiles * 256 * 2;
-            const long long t_single = (long long)s_cost[3] * n_col_tiles * kTileNUmma;
-            use_pair = (pair.force || (min(mean, (long long)s_pair_min) >= kPairMinUnits &&
-                                       t_pair * 100 <= t_single * kPairAdvantagePct)) ? 1 : 0;
+            const long long t_single = (long long)s_cost[3] * n_col_tiles * pair.single_cols;
+            const long long u = min(mean, (long long)s_pair_min);
+            use_pair = (pair.force || t_pair * (u + kPairDrainUnits) * 100 <= t_single * (u + kPieceChargeUnits) * kPairAdvantagePct) ? 1 : 0;
         }
         plan->pad[0] = use_pair;                      // which tensor-core core runs: 1 = the two-SM core
         plan->pad[1] = charge;                        // virtual units in front of every (row tile, column tile) in the prefix sums
@@ -237,15 +240,16 @@ plan_finish_kernel(int32_t n_row_tiles, int32_t n_col_tiles, int32_t target_item
 {
     __shared__ unsigned long long s_cost[64];
     __shared__ int32_t s_scan[34];
-    finish_plan(n_row_tiles, n_col_tiles, target_items, wave_ctas, planes_per_len, plan, scratch, s_cost, s_scan, PairChoice{0, 0, 0});
+    finish_plan(n_row_tiles, n_col_tiles, target_items, wave_ctas, planes_per_len, plan, scratch, s_cost, s_scan, PairChoice{0, 0, 0, kTileNUmma});
 }
 
 cudaError_t launch_plan(const int32_t *L, int64_t M, int32_t group, int32_t Lmax, int64_t kw, int ppq, int64_t m_pad,
                         int64_t n_col_tiles, int32_t target_items, int32_t wave_ctas, int32_t *l_rows,
                         int32_t *perm, int32_t *l_sorted, PlanHeader *plan, int32_t *scratch, cudaStream_t st,
-                        int64_t batch, int32_t pos_block, int32_t pair_col_tiles, int32_t pair_clusters, int32_t pair_force)
+                        int64_t batch, int32_t pos_block, int32_t pair_col_tiles, int32_t pair_clusters, int32_t pair_force,
+                        int32_t single_tile_cols)
 {
-    const PairChoice pair{pair_col_tiles, batch == 1 ? pair_clusters : 0, pair_force};
+    const PairChoice pair{pair_col_tiles, batch == 1 ? pair_clusters : 0, pair_force, single_tile_cols};
     if (batch < 1 || batch > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
     plan_kernel<<<(unsigned)batch, kPlanThreads, 0, st>>>(L, M, group, Lmax, (int32_t)(kw * ppq), pos_block, m_pad, (int32_t)n_col_tiles,
                                                         target_items, wave_ctas, l_rows, perm, l_sorted, plan, scratch, pair);
