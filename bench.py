@@ -360,7 +360,9 @@ def run_attention(args):
         binding.sc_profile_enable(sc.ctx, False)
         bitops = float(B) * M * N * K * w.L
         t, tc = min(step_ms) * 1e-3, min(core_ms) * 1e-3
-        pad = (round_up(M, 128) * round_up(N, 192)) / float(M * N)
+        tiles = (N + 191) // 192                              # the one-SM tensor-core core spreads N evenly over its tiles,
+        tile_n = min(192, round_up((N + tiles - 1) // tiles, 32))   # in multiples of 32 columns
+        pad = (round_up(M, 128) * tiles * tile_n) / float(M * N)
         rows.append((w.name, B, M, K, N, w.mode, w.L, bitops, t * 1e3, bitops / t, tc * 1e3, bitops / tc, pad))
         del A, W, C
     assert sc.device_status() == 0

@@ -327,10 +327,13 @@ size_t sc_workspace_bytes(int64_t M, int64_t K, int64_t N, int32_t Lmax, const s
 
 // Padding of the output columns of one product: a single product is padded for every core (prepared weights may be
 // used by either family); stacked products only for the core that will run, which keeps narrow products small.
-static int64_t batched_col_pad(const sc_params *p, int64_t K, int32_t Lmax, int64_t B)
+static int64_t batched_col_pad(const sc_params *p, int64_t K, int32_t Lmax, int64_t B, int64_t N)
 {
     if (B <= 1) return kColPad;
-    return pick_variant(p, K, Lmax) == SC_CORE_UMMA ? kTileNUmma : kTileN;
+    if (pick_variant(p, K, Lmax) != SC_CORE_UMMA) return kTileN;
+    // the tensor-core core's own tiles: its column tile follows N (umma_tile_cols), and a product takes exactly its tiles
+    const int64_t tile_n = umma_tile_cols(N);
+    return (N + tile_n - 1) / tile_n * tile_n;
 }
 
 // Shared body of sc_matmul (W given, everything derived per call) and sc_matmul_prepared (pw given).
@@ -346,7 +349,7 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     if (B * round_up(M, kTileM) >= (1LL << 24) || B * round_up(N, kColPad) >= (1LL << 24)) return SC_ERR_SHAPE;
     if (Lmax < 1 || Lmax > SC_L_CAP || (int64_t)K * Lmax >= (1LL << 30)) return SC_ERR_LENGTH;
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return SC_ERR_WORKSPACE;
-    const int64_t col_pad = batched_col_pad(params, K, Lmax, B);
+    const int64_t col_pad = batched_col_pad(params, K, Lmax, B, N);
     const Workspace w = layout_workspace(M, K, N, Lmax, params->mode, P == nullptr, pw == nullptr, B, col_pad);
     if (ws_bytes < w.total) return SC_ERR_WORKSPACE;
     if (params->core == SC_CORE_SIMPLE && (B == 1 ? M : w.m_pad) > 65535) return SC_ERR_SHAPE;
@@ -509,7 +512,7 @@ sc_status sc_matmul(sc_ctx *ctx, const float *A, const float *W, int64_t M, int6
 size_t sc_workspace_bytes_batched(int64_t B, int64_t M, int64_t K, int64_t N, int32_t Lmax, const sc_params *params)
 {
     if (!params_ok(params) || B < 1 || B > 65535 || M <= 0 || K <= 0 || N <= 0 || Lmax < 1 || Lmax > SC_L_CAP) return 0;
-    return layout_workspace(M, K, N, Lmax, params->mode, true, true, B, batched_col_pad(params, K, Lmax, B)).total;
+    return layout_workspace(M, K, N, Lmax, params->mode, true, true, B, batched_col_pad(params, K, Lmax, B, N)).total;
 }
 
 sc_status sc_matmul_batched(sc_ctx *ctx, const float *A, const float *W, int64_t B, int64_t M, int64_t K, int64_t N,
