@@ -123,6 +123,23 @@ def test_int8_grid_first_quantisation(sc, binding, oracle, mode):
     binding.sc_weights_release(prepared[0])
 
 
+@pytest.mark.parametrize("mode", ["bipolar", "unipolar"])
+@pytest.mark.parametrize("M,N", [(1100, 523), (1024, 512)])
+def test_sm_pair_core_odd_tiles_and_ragged_edges(sc, binding, oracle, mode, M, N):
+    """The two-SM tensor-core core on shapes that stress its tiling: nine row tiles (the last pair has one tile only), a last
+    column tile of 11 columns with N not a multiple of 4 (no bulk reductions), lengths from 0 upwards with whole tiles of
+    finished rows; and the exact-fit shape.  Every entry against the oracle."""
+    w, L_rows = wl.small_ragged(seed=91, M=M, K=100, N=N, mode=mode, Lmin=0, Lmax=56)
+    L_rows[:5] = [56, 0, 1, 55, 56]
+    L_rows[M // 2:M // 2 + 300] = 0                    # more than two tiles of rows without a stream
+    A, W = wl.make_inputs(w)
+    P, C = T.gpu_matmul(sc, binding, w, A, W, L_rows, 56, core=5)
+    ref = T.oracle_matmul(oracle, w, A, W, L_rows)
+    assert np.array_equal(P, ref["P"])
+    assert T.close_enough(C, ref["C"])
+    assert sc.device_status() == 0
+
+
 def test_groups_and_accumulator_workspace(sc, binding, oracle):
     """Lengths per group of 8 rows (last group short); P not requested (accumulators live in the workspace)."""
     w, _ = wl.small_ragged(seed=5, M=150, K=96, N=130)
