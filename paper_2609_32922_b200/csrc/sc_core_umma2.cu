@@ -94,11 +94,17 @@ __device__ __forceinline__ void p_cluster_sync()
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// arrive on the barrier at the same shared-memory offset in CTA `cta` of the pair (release at cluster scope)
+// Arrive on the barrier at the same shared-memory offset in CTA `cta` of the pair: the plain form, a release at CTA scope.
+// What the arrival hands over never needs more.  Operand A and the accumulators live in tensor memory, ordered by
+// tcgen05.wait and tcgen05.fence::before_thread_sync.  Operand W is written by ordinary stores to the ARRIVING CTA's own
+// shared memory and published to the async proxy by fence.proxy.async before the arrival; the two-SM MMA reads each CTA's
+// half of W from that CTA's own shared memory, so the leader's issuing thread passes on only the barrier's phase.  A release
+// at cluster scope would add a fence that costs each expander warp a round trip beyond the SM per stage: measured, 13 - 20 %
+// of the kernel's time, all of it on the W side, which is the critical path.
 __device__ __forceinline__ void p_arrive_cta(uint32_t bar, uint32_t cta)
 {
     asm volatile("{\n\t.reg .b32 ra;\n\tmapa.shared::cluster.u32 ra, %0, %1;\n\t"
-                 "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}" ::"r"(bar), "r"(cta) : "memory");
+                 "mbarrier.arrive.shared::cluster.b64 _, [ra];\n\t}" ::"r"(bar), "r"(cta) : "memory");
 }
 __device__ __forceinline__ void p_store_cta(uint32_t addr, uint32_t cta, uint32_t value)
 {
@@ -445,7 +451,7 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
                     n_act = min(x.my_len - pp0 / (kPosBlockSigned * ppl) * kPosBlockSigned, x.q1 - pp0);
                 }
 #pragma unroll
-                for (int q = 0; q < kPStagePp; ++q) dst[q] = q < n_act ? __ldcs(x.src + (int64_t)q * p.m_pad) : 0u;
+                for (int q = 0; q < kPStagePp; ++q) dst[q] = q < n_act ? __ldg(x.src + (int64_t)q * p.m_pad) : 0u;
                 if (a_signed) {
                     uint4 v = make_uint4(0u, 0u, 0u, 0u);
                     if (n_act > 0) {
@@ -489,19 +495,26 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
                 it.op = (uint32_t)(group - kPAGroups); it.j = group - kPAGroups; it.src += (int64_t)(group - kPAGroups) * stage_stride;
                 advance(it);
             }
-            // two register sets take turns: while one is expanded, the words of the group's next stage land in the other
+            // Two register sets take turns.  The words of a stage are requested right AFTER the group's previous hand-over and
+            // used two hand-overs later: a hand-over (the release of the barrier arrival) waits for the thread's loads in
+            // flight, so loads issued just before it would hold it up for most of their latency (measured: a quarter of the
+            // expander's time), and this way they have a whole period of the group to land.
             uint32_t w0[kPStagePp], w1[kPStagePp], s0[kSignWords], s1[kSignWords];
             uint32_t op0 = it.op, op1 = 0u;
             bool v0 = it.valid, v1 = false;
             if (v0) { fetch(it, w0, s0); advance(it); }
+            v1 = it.valid; op1 = it.op;
+            if (v1) { fetch(it, w1, s1); advance(it); }
             while (v0 && ok && !*s_abort) {
-                v1 = it.valid; op1 = it.op;
-                if (v1) { fetch(it, w1, s1); advance(it); }
                 process(w0, s0, op0);
-                if (!ok || !v1 || *s_abort) { op0 = op1; break; }
+                if (!ok || *s_abort) break;
                 v0 = it.valid; op0 = it.op;
                 if (v0) { fetch(it, w0, s0); advance(it); }
+                if (!v1) break;
                 process(w1, s1, op1);
+                if (!ok || *s_abort) break;
+                v1 = it.valid; op1 = it.op;
+                if (v1) { fetch(it, w1, s1); advance(it); }
             }
             if (!ok && lane == 0) give_up(7, op0, op1);
         };
