@@ -132,6 +132,25 @@ __device__ __forceinline__ bool p_mbar_wait_cluster(uint32_t bar, uint32_t parit
         }
     }
 }
+// The same wait by a whole warp on the four consecutive barriers from `bar0` at once: lane k polls barrier k % 4, so the four
+// polls are one instruction and their latencies overlap.  (Polled one after the other by one thread they cost about 350 clocks
+// each even when complete, which made the issuing threads the bottleneck of the kernel.)  Uniform result.
+__device__ __forceinline__ bool p_mbar_wait4_warp(uint32_t bar0, uint32_t parity, volatile int32_t *abort_flag, int lane)
+{
+    const uint32_t mine = bar0 + 8u * (uint32_t)(lane & 3);
+    long long t0 = 0;
+    for (uint32_t spins = 1;; ++spins) {
+        const bool done = p_mbar_try_cluster(mine, parity);
+        if (__all_sync(0xFFFFFFFFu, done)) return true;
+        if ((spins & 63u) == 0u) {
+            bool stop = *abort_flag != 0;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kUWaitCycles) stop = true;
+            if (__any_sync(0xFFFFFFFFu, stop)) return false;
+        }
+    }
+}
 // D[tmem of both CTAs] (+)= A[tmem of both CTAs] x B[shared memory of both CTAs], 256 x 256 x 64
 __device__ __forceinline__ void p_mma_fp4_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate,
                                              uint32_t sfa_tmem, uint32_t sfb_tmem)
@@ -290,10 +309,12 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
             if (!ok) give_up(1, raw_cnt, 0);
         }
     } else if (warp == 1 || warp >= kPIssuerBWarp) {
-        // ---------------- MMA issuers (leader CTA): issuer i owns the ring slots s with s % 2 == i ----------------
-        if (lane == 0 && rank == 0) {
+        // ---------------- MMA issuers (leader CTA): issuer i owns the stages n with n % kPIssuers == i ----------------
+        // The whole warp walks the pieces and polls (one barrier per lane); lane 0 issues.  The path of an issuer per stage is
+        // kept short: it, not the tensor pipe, bounds the kernel as soon as it takes longer than kPIssuers stages of MMAs.
+        if (rank == 0) {
             const uint32_t me = warp == 1 ? 0u : (uint32_t)(warp - kPIssuerBWarp + 1);
-            uint32_t op_cnt = 0, acc_cnt = 0;
+            uint32_t op_cnt = 0, acc_cnt = 0;                     // stages / pieces before the current piece
             bool ok = true;
             int site = 0;
             const uint64_t desc0 = u_smem_desc(ops_addr, kPLbo);
@@ -305,38 +326,45 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
                 const uint32_t acc_phase = acc_cnt & 1u;
                 const uint32_t first = op_cnt % kPIssuers;        // owner of the piece's first stage: it overwrites
                 site = 2;
-                ok = p_mbar_wait_cluster(bar(kPAccEmpty), acc_phase ^ 1u, s_abort);
-                if (ok && me != first) { site = 3; ok = u_mbar_wait(bar(kPAccStarted), acc_phase, s_abort); }
+                {
+                    int good = 1;
+                    if (lane == 0) good = p_mbar_wait_cluster(bar(kPAccEmpty), acc_phase ^ 1u, s_abort) ? 1 : 0;
+                    ok = __shfl_sync(0xFFFFFFFFu, good, 0) != 0;
+                }
+                if (ok && me != first) { site = 3; ok = u_mbar_wait_warp(bar(kPAccStarted), acc_phase, s_abort, lane); }
                 if (!ok) break;
                 site = 4;
                 const int32_t n_ops = it.n_raw * kPOpsPerRaw;
-                bool issued_any = false;
-                for (int32_t j = 0; j < n_ops; ++j, ++op_cnt) {
-                    if (op_cnt % kPIssuers != me) continue;
-                    const uint32_t t = op_cnt % kPOpStages;
-                    for (int k = 0; k < 4 && ok; ++k)
-                        ok = p_mbar_wait_cluster(bar(kPOpFull + 4 * t + k), (op_cnt / kPOpStages) & 1u, s_abort);
+                const int32_t j0 = (int32_t)((me + kPIssuers - first) % kPIssuers);
+                for (int32_t j = j0; j < n_ops; j += kPIssuers) {
+                    const uint32_t op = op_cnt + (uint32_t)j;
+                    const uint32_t t = op % kPOpStages, use = op / kPOpStages;
+                    ok = p_mbar_wait4_warp(bar(kPOpFull + 4 * t), use & 1u, s_abort, lane);
                     if (!ok) break;
                     u_fence_after();
-                    const uint64_t bdesc = desc0 + (uint64_t)(t * kStageDesc);
-                    const uint32_t a_base = tmem_base + kPARingCol + t * (kPOpSteps * 8u);
+                    if (lane == 0) {
+                        const uint64_t bdesc = desc0 + (uint64_t)(t * kStageDesc);
+                        const uint32_t a_base = tmem_base + kPARingCol + t * (kPOpSteps * 8u);
 #pragma unroll
-                    for (int st = 0; st < kPOpSteps; ++st) {
-                        p_mma_fp4_ts(tmem_base, a_base + st * 8u, bdesc + (uint64_t)(st * kStepDesc), idesc,
-                                     (uint32_t)((j | st) != 0), tmem_base + kPSfCol, tmem_base + kPSfCol + 32u);
-                        if (j == 0 && st == 0) u_mbar_arrive(bar(kPAccStarted));       // the overwrite is in the pipe
+                        for (int st = 0; st < kPOpSteps; ++st) {
+                            p_mma_fp4_ts(tmem_base, a_base + st * 8u, bdesc + (uint64_t)(st * kStepDesc), idesc,
+                                         (uint32_t)((j | st) != 0), tmem_base + kPSfCol, tmem_base + kPSfCol + 32u);
+                            if (j == 0 && st == 0) u_mbar_arrive(bar(kPAccStarted));       // the overwrite is in the pipe
+                        }
+                        // frees the ring slot in both CTAs when these MMAs have read it (even and odd uses of a slot signal
+                        // barriers of their own)
+                        p_commit_pair(bar(kPOpEmpty + t + kPOpStages * (use & 1u)));
                     }
-                    issued_any = true;
-                    // frees the ring slot in both CTAs when these MMAs have read it (even and odd uses of a slot signal
-                    // barriers of their own)
-                    p_commit_pair(bar(kPOpEmpty + t + kPOpStages * ((op_cnt / kPOpStages) & 1u)));
                 }
                 if (!ok) break;
-                if (issued_any) p_commit_pair(bar(kPAccFull));    // this issuer's share of the accumulators is complete
-                else { p_arrive_cta(bar(kPAccFull), 0u); p_arrive_cta(bar(kPAccFull), 1u); }      // (no stage of its own in this piece)
+                if (lane == 0) {
+                    if (j0 < n_ops) p_commit_pair(bar(kPAccFull));    // this issuer's share of the accumulators is complete
+                    else { p_arrive_cta(bar(kPAccFull), 0u); p_arrive_cta(bar(kPAccFull), 1u); }      // (no stage of its own in this piece)
+                }
+                op_cnt += (uint32_t)n_ops;
                 ++acc_cnt;
             }
-            if (!ok) give_up(site, op_cnt, acc_cnt);
+            if (!ok && lane == 0) give_up(site, op_cnt, acc_cnt);
         }
     } else if (warp < kPAFirstWarp) {
         // ---------------- epilogue: this CTA's 128 rows of the 256 x 256 accumulator ----------------
