@@ -112,7 +112,7 @@ static bool choose_pair(sc_ctx_impl *c, const sc_params *params, bool umma, int6
     if (pair_core_clusters(params->mode, c->sm_count, &out->clusters) != cudaSuccess) return false;
     if (out->clusters < 1) out->mode = 0;
     if (out->mode == 1) {
-        // The plan selects the two-SM core only if its tiling costs at most 28 % more MMA time than the one-SM core's (its
+        // The plan selects the two-SM core only if its tiling costs at most 50 % more MMA time than the one-SM core's (its
         // measured advantage on long pieces; shorter pieces tighten the condition).  Where the shape alone already rules
         // that out (an odd row tile, a ragged last column tile: ragged lengths only add to it), the two-SM kernel is not
         // enqueued at all.
@@ -120,7 +120,7 @@ static bool choose_pair(sc_ctx_impl *c, const sc_params *params, bool umma, int6
         const int64_t t_pair = pairs * out->col_tiles * pair_core_tile_cols() * 2;
         const int64_t tile_n = umma_tile_cols(N);
         const int64_t t_single = row_tiles * ((N + tile_n - 1) / tile_n) * tile_n;
-        if (t_pair * 100 > t_single * 128) out->mode = 0;
+        if (t_pair * 100 > t_single * 150) out->mode = 0;
     }
     return true;
 }

@@ -327,29 +327,29 @@ core_umma_kernel(const __grid_constant__ CUtensorMap map_w, UmmaDev p)
                 site = 4;
                 const uint32_t d_tmem = tmem_base + b * kAccCols;
                 const int32_t n_ops = it.n_raw * kOpsPerRaw;
-                bool issued_any = false;
-                for (int32_t j = 0; j < n_ops; ++j, ++op_cnt) {
-                    if (op_cnt % kIssuers != me) continue;
-                    const uint32_t t = op_cnt % kOpStages;
-                    ok = u_mbar_wait(bar(kOpFull + t), (op_cnt / kOpStages) & 1u, s_abort);
+                const int32_t j0 = (int32_t)((me + kIssuers - first) % kIssuers);      // the issuer's first stage of the item
+                for (int32_t j = j0; j < n_ops; j += kIssuers) {
+                    const uint32_t op = op_cnt + (uint32_t)j;
+                    const uint32_t t = op % kOpStages, use = op / kOpStages;
+                    ok = u_mbar_wait(bar(kOpFull + t), use & 1u, s_abort);
                     if (!ok) break;
                     u_fence_after();
                     const uint64_t bdesc = desc0 + (uint64_t)(t * kStageDesc);
-                    const uint32_t a_base = tmem_base + a_ring_col + a_slot(op_cnt) * (kOpSteps * 8u);
+                    const uint32_t a_base = tmem_base + a_ring_col + a_slot(op) * (kOpSteps * 8u);
 #pragma unroll
                     for (int st = 0; st < kOpSteps; ++st) {
                         u_mma_fp4_ts(d_tmem, a_base + st * 8u, bdesc + (uint64_t)(st * kStepDesc), idesc,
                                      (uint32_t)((j | st) != 0), tmem_base + kSfCol, tmem_base + kSfCol + 16u);
                         if (j == 0 && st == 0) u_mbar_arrive(bar(kAccStarted + b));     // the overwrite is in the pipe
                     }
-                    issued_any = true;
                     // frees the operand stage when these MMAs have read it (even and odd uses of a stage have
                     // barriers of their own)
-                    u_commit(bar(kOpEmpty + t + kOpStages * ((op_cnt / kOpStages) & 1u)));
+                    u_commit(bar(kOpEmpty + t + kOpStages * (use & 1u)));
                 }
                 if (!ok) break;
-                if (issued_any) u_commit(bar(kAccFull + b));     // this issuer's share of the accumulator is complete
+                if (j0 < n_ops) u_commit(bar(kAccFull + b));     // this issuer's share of the accumulator is complete
                 else u_mbar_arrive(bar(kAccFull + b));           // (it had no stage in this item)
+                op_cnt += (uint32_t)n_ops;
                 ++acc_cnt;
             }
             if (!ok) give_up(site, op_cnt, acc_cnt);

@@ -11,13 +11,13 @@ constexpr int kPlanThreads = 1024;
 
 // Two-SM core (sc_core_umma2.cu): it has one accumulator, so a piece boundary drains its pipeline (about kPairDrainUnits stage
 // units, against the kPieceChargeUnits of the one-SM core), it works on pairs of row tiles and on 256-column tiles (an odd row
-// tile or a ragged last column tile is padding), and on long pieces it needs 22 % less time per multiply-accumulate.  It is
+// tile or a ragged last column tile is padding), and on long pieces it needs a third less time per multiply-accumulate.  It is
 // selected when its estimated time is the shorter one:
-//     t_pair (u + kPairDrainUnits) <= 1.28 t_single (u + kPieceChargeUnits),   u = min(mean units per piece, shortest tile pair),
+//     t_pair (u + kPairDrainUnits) <= 1.50 t_single (u + kPieceChargeUnits),   u = min(mean units per piece, shortest tile pair),
 // t = stage units x column tiles x tile columns / SMs per tile (MMA time up to a common factor).  Measured against the forced
 // choices on the ViT-L/14 sweep and the ragged configurations (profiles/core_umma_pair_kernel_*.md).
-constexpr long long kPairDrainUnits = 15;
-constexpr long long kPairAdvantagePct = 128;       // break-even near 35 units per piece on unpadded shapes
+constexpr long long kPairDrainUnits = 20;
+constexpr long long kPairAdvantagePct = 150;       // break-even near 28 units per piece on unpadded shapes
 // One-SM tensor-core core: a piece boundary costs about this many stage units (accumulator hand-over, pipeline refill); the
 // prefix sums charge it to every (row tile, column tile) so that equal runs are runs of equal time (see u_piece).
 constexpr int32_t kPieceChargeUnits = 4;      // measured: 0 / 4 / 8 / 12 units give 0.120 / 0.117 / 0.117 / 0.121 ms on the per-row mixed
