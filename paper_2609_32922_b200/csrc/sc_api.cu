@@ -102,7 +102,8 @@ struct PairLaunch {
     int clusters;           // CTA pairs the two-SM kernel runs with
     int32_t col_tiles;      // its column tiles
 };
-static bool choose_pair(sc_ctx_impl *c, const sc_params *params, bool umma, int64_t m_pad, int64_t N, int64_t B, PairLaunch *out)
+static bool choose_pair(sc_ctx_impl *c, const sc_params *params, bool umma, int64_t m_pad, int64_t N, int64_t B, int64_t max_units,
+                        PairLaunch *out)
 {
     out->mode = 0;
     out->clusters = 0;
@@ -113,14 +114,15 @@ static bool choose_pair(sc_ctx_impl *c, const sc_params *params, bool umma, int6
     if (out->clusters < 1) out->mode = 0;
     if (out->mode == 1) {
         // The plan selects the two-SM core only if its tiling costs at most 50 % more MMA time than the one-SM core's (its
-        // measured advantage on long pieces; shorter pieces tighten the condition).  Where the shape alone already rules
-        // that out (an odd row tile, a ragged last column tile: ragged lengths only add to it), the two-SM kernel is not
-        // enqueued at all.
+        // measured advantage on long pieces; shorter pieces tighten the condition).  Where the shape and Lmax alone already
+        // rule that out (an odd row tile, a ragged last column tile, short streams: ragged lengths only add to it), the two-SM
+        // kernel is not enqueued at all.
         const int64_t row_tiles = m_pad / kTileM, pairs = (row_tiles + 1) / 2;
         const int64_t t_pair = pairs * out->col_tiles * pair_core_tile_cols() * 2;
         const int64_t tile_n = umma_tile_cols(N);
         const int64_t t_single = row_tiles * ((N + tile_n - 1) / tile_n) * tile_n;
-        if (t_pair * 100 > t_single * 150) out->mode = 0;
+        // (max_units: stage units of the longest possible piece, from Lmax; shorter pieces only tighten the condition)
+        if (t_pair * (max_units + kPairDrainUnits) * 100 > t_single * (max_units + kPieceChargeUnits) * kPairAdvantagePct) out->mode = 0;
     }
     return true;
 }
@@ -388,7 +390,8 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     uint32_t *a_sign = reinterpret_cast<uint32_t *>(base + w.a_sign);
     const bool signs = umma && params->mode == SC_UNIPOLAR_AND;
     PairLaunch pair;
-    if (!choose_pair(c, params, umma, w.m_pad, N, B, &pair)) return SC_ERR_CUDA;
+    const int64_t l_round = params->mode == SC_UNIPOLAR_AND ? round_up(Lmax, kPosBlockSigned) : Lmax;
+    if (!choose_pair(c, params, umma, w.m_pad, N, B, (l_round * w.kw + kStagePlanes - 1) / kStagePlanes, &pair)) return SC_ERR_CUDA;
     const int pair_mode = pair.mode, pair_clusters = pair.clusters;
     const int32_t pair_col_tiles = pair.col_tiles;
 
@@ -580,7 +583,7 @@ sc_status sc_matmul_cbsg(sc_ctx *ctx, const float *A, const float *W, int64_t M,
     const int32_t tile_n = umma_tile_cols(N);
     const int64_t n_col_tiles = (N + tile_n - 1) / tile_n;
     PairLaunch pair;
-    if (!choose_pair(c, params, true, w.m_pad, N, 1, &pair)) return SC_ERR_CUDA;
+    if (!choose_pair(c, params, true, w.m_pad, N, 1, ((int64_t)core_lmax * w.kw + kStagePlanes - 1) / kStagePlanes, &pair)) return SC_ERR_CUDA;
     if (launch_plan(l_core, M, params->group, core_lmax, w.kw, 1, w.m_pad, n_col_tiles, 0, c->sm_count, l_rows,
                     perm, l_sorted, plan, c->scratch, st, 1, 1, pair.col_tiles, pair.mode ? pair.clusters : 0,
                     pair.mode == 2, tile_n) != cudaSuccess)

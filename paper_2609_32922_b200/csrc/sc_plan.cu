@@ -16,12 +16,8 @@ constexpr int kPlanThreads = 1024;
 //     t_pair (u + kPairDrainUnits) <= 1.50 t_single (u + kPieceChargeUnits),   u = min(mean units per piece, shortest tile pair),
 // t = stage units x column tiles x tile columns / SMs per tile (MMA time up to a common factor).  Measured against the forced
 // choices on the ViT-L/14 sweep and the ragged configurations (profiles/core_umma_pair_kernel_*.md).
-constexpr long long kPairDrainUnits = 20;
-constexpr long long kPairAdvantagePct = 150;       // break-even near 28 units per piece on unpadded shapes
-// One-SM tensor-core core: a piece boundary costs about this many stage units (accumulator hand-over, pipeline refill); the
-// prefix sums charge it to every (row tile, column tile) so that equal runs are runs of equal time (see u_piece).
-constexpr int32_t kPieceChargeUnits = 4;      // measured: 0 / 4 / 8 / 12 units give 0.120 / 0.117 / 0.117 / 0.121 ms on the per-row mixed
-                                              // ViT-B/16 qkv configuration and 2.03 / 1.94 / 1.96 / 1.99 ms on the grouped DiT-like one
+// (kPairDrainUnits, kPairAdvantagePct, kPieceChargeUnits: sc_internal.h; the host applies the same rule to the longest
+// possible piece to decide whether the two-SM kernel is enqueued at all.)
 
 struct PairChoice {
     int32_t col_tiles;      // column tiles of the two-SM core (0: that core is not available for the call)
