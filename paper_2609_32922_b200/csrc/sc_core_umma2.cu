@@ -168,6 +168,7 @@ __device__ __forceinline__ void p_commit_pair(uint32_t bar)
 
 struct PItem {
     int32_t pair, ct, q0, q1, n_raw;
+    bool whole;             // the piece is the whole (tile pair, column tile): nothing else adds to these outputs
 };
 
 // stage units of a pair per column tile: the longer (first) row tile of the pair decides
@@ -192,6 +193,7 @@ __device__ __forceinline__ PItem p_piece(const int32_t *s_prefix, int32_t n_pair
     it.q0 = s0 * kStagePlanes;
     it.q1 = min(s1 * kStagePlanes, planes);
     it.n_raw = s1 - s0;
+    it.whole = s0 == 0 && s1 == stages;
     (void)n_col_tiles;
     return it;
 }
@@ -395,7 +397,23 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
                     uint32_t *buf = tile0 + (chunk_cnt & 1u) * (32 * kPEpiStride);
                     asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");     // the buffer's previous reduction has read it
                     const int64_t col0 = (int64_t)it.ct * kPN + c * 32;
-                    if (bulk_ok && col0 + 32 <= p.N) {
+                    if (it.whole) {
+                        // No other piece adds to this tile: the zeroed outputs are simply overwritten, straight from the
+                        // registers (eight 16-byte stores per row piece; a dozen instructions per chunk).  With one accumulator
+                        // the MMAs wait for the epilogue, and the bulk reduction below costs the warp about 2000 clocks per chunk.
+                        if (src >= 0) {
+                            int32_t *row = p.acc + (int64_t)src * p.N + col0;
+                            if (bulk_ok && col0 + 32 <= p.N) {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    reinterpret_cast<uint4 *>(row)[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                            } else {
+#pragma unroll
+                                for (int k = 0; k < 32; ++k)
+                                    if (col0 + k < p.N) row[k] = (int32_t)v[k];
+                            }
+                        }
+                    } else if (bulk_ok && col0 + 32 <= p.N) {
                         uint4 *dst = reinterpret_cast<uint4 *>(buf + lane * kPEpiStride);
 #pragma unroll
                         for (int j = 0; j < 8; ++j) dst[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
