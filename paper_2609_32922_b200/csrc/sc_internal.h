@@ -27,11 +27,11 @@ inline int umma_tile_cols(int64_t N)
 constexpr int kStagePlanes = 16;     // stream planes per pipeline stage
 // Selection between the two tensor-core kernels (sc_plan.cu states the rule): a piece boundary of the two-SM core costs
 // about kPairDrainUnits stage units, one of the one-SM core kPieceChargeUnits; on long pieces the two-SM core needs
-// 100 / kPairAdvantagePct of the one-SM core's time per multiply-accumulate (break-even near 28 units per piece on unpadded
+// 100 / kPairAdvantagePct of the one-SM core's time per multiply-accumulate (break-even near 16 units per piece on unpadded
 // shapes).  kPieceChargeUnits is also what the prefix sums charge every (row tile, column tile) of the one-SM core; measured:
 // 0 / 4 / 8 / 12 units give 0.120 / 0.117 / 0.117 / 0.121 ms on the per-row mixed ViT-B/16 qkv configuration and
 // 2.03 / 1.94 / 1.96 / 1.99 ms on the grouped DiT-like one.
-constexpr long long kPairDrainUnits = 20;
+constexpr long long kPairDrainUnits = 14;
 constexpr long long kPairAdvantagePct = 150;
 constexpr int kPieceChargeUnits = 4;
 constexpr int kStages = 4;           // TMA pipeline depth
