@@ -140,6 +140,27 @@ def test_sm_pair_core_odd_tiles_and_ragged_edges(sc, binding, oracle, mode, M, N
     assert sc.device_status() == 0
 
 
+@pytest.mark.parametrize("N", [1024, 1022])
+def test_sm_pair_core_whole_tile_pieces(sc, binding, oracle, N):
+    """The two-SM core when its pieces are whole tiles (148 equal tiles on 74 CTA pairs: every run ends on a tile edge), which
+    overwrite the zeroed outputs with plain stores instead of reductions: 16-byte stores (N = 1024) and, with N not a multiple
+    of 4, single-word stores with a ragged last column tile.  A few rows without a stream shorten the last tile, so that some
+    pieces are cut there and both epilogue paths meet in one call.  Every entry against the oracle."""
+    M = 37 * 256
+    w, L_rows = wl.small_ragged(seed=17, M=M, K=32, N=N, mode="bipolar", Lmin=8, Lmax=8)
+    L_rows[:] = 8
+    A, W = wl.make_inputs(w)
+    for zero_rows in (0, 40):
+        L = L_rows.copy()
+        if zero_rows:
+            L[100:100 + zero_rows] = 0
+        P, C = T.gpu_matmul(sc, binding, w, A, W, L, 8, core=5)
+        ref = T.oracle_matmul(oracle, w, A, W, L)
+        assert np.array_equal(P, ref["P"])
+        assert T.close_enough(C, ref["C"])
+    assert sc.device_status() == 0
+
+
 def test_groups_and_accumulator_workspace(sc, binding, oracle):
     """Lengths per group of 8 rows (last group short); P not requested (accumulators live in the workspace)."""
     w, _ = wl.small_ragged(seed=5, M=150, K=96, N=130)
