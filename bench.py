@@ -674,11 +674,14 @@ def main():
         peak_b = 2.0 * mac_per_clk_sm * n_sm * sm_max * 1e6 / 1e12
         peak_tops = max(peak_a, peak_b)
         ach = 2.0 * achieved / 1e12
+        pair_ran = binding.sc_last_core_selected(sc.ctx) != 0          # the plan's choice between the two tensor-core kernels
         roofline = {
             "bound": "tensor",
-            "kernel": "core_umma_kernel (tcgen05.mma kind::mxf4 on bits expanded on chip)",
+            "kernel": ("core_umma_pair_kernel (tcgen05.mma.cta_group::2 kind::mxf4, 256 x 256 tiles on pairs of SMs, bits "
+                       "expanded on chip)" if pair_ran else
+                       "core_umma_kernel (tcgen05.mma kind::mxf4 on bits expanded on chip)"),
             "achieved": ach, "peak": peak_tops, "unit": "TFLOP/s", "frac": ach / peak_tops,
-            "traffic": NCU_CORE_TRAFFIC_BYTES.get((w.name, "umma")),
+            "traffic": NCU_CORE_TRAFFIC_BYTES.get((w.name, "pair" if pair_ran else "umma")),
             "peak_source": ("the larger of (a) %s x %g (nominal fp4 : bf16) = %.0f TFLOP/s and (b) measured issue rate of "
                             "the mxf4 MMA, %.0f MAC/clk/SM x %d SMs x %.0f MHz = %.0f TFLOP/s"
                             % ("measured bf16 burst %.1f TFLOP/s (MEASURED_PEAKS.json)" % bf16 if bf16

@@ -278,6 +278,11 @@ sc_status sc_profile_read(sc_ctx *ctx, float *ms_out /* HOST [SC_PROFILE_PHASES]
 /* Number of kernels this library has launched through `ctx` since sc_create (memsets not counted). */
 sc_status sc_launch_count(sc_ctx *ctx, int64_t *count_host);
 
+/* Which tensor-core kernel the most recent sc_matmul / sc_matmul_prepared / sc_matmul_cbsg call through `ctx` selected
+ * (the choice is made on the device from the stream lengths): *pair_host = 1 the two-SM kernel (SC_CORE_UMMA_PAIR),
+ * 0 the one-SM kernel or a call that ran on the integer cores.  Synchronises on the device.  `pair_host`: HOST.       */
+sc_status sc_last_core_selected(sc_ctx *ctx, int32_t *pair_host);
+
 /* ---- host-side self checks and device micro-benchmarks ---------------------------------------- */
 /* Exhaustive host check of the bit-plane comparator used by the encode kernel against r < T for all
  * 257 boundaries and 256 draws; returns the number of mismatches (0 = correct).  Runs on the CPU.   */

@@ -24,7 +24,7 @@ SC_L_CAP = 1024
 EXPORTS = (
     "sc_create", "sc_destroy", "sc_status_string", "sc_device_status", "sc_row_stats", "sc_assign_lengths",
     "sc_ladder_lengths", "sc_stream_bytes", "sc_encode", "sc_debug_unpack", "sc_workspace_bytes", "sc_matmul",
-    "sc_selftest_comparator", "sc_selftest_expansion", "sc_selftest_bounded_wait", "sc_microbench", "sc_profile_enable", "sc_profile_read", "sc_launch_count",
+    "sc_selftest_comparator", "sc_selftest_expansion", "sc_selftest_bounded_wait", "sc_microbench", "sc_profile_enable", "sc_profile_read", "sc_launch_count", "sc_last_core_selected",
     "sc_assign_lengths_static", "sc_weights_bytes", "sc_weights_prepare", "sc_weights_release",
     "sc_workspace_bytes_prepared", "sc_matmul_prepared", "sc_surrogate_noise",
     "sc_workspace_bytes_batched", "sc_matmul_batched", "sc_workspace_bytes_cbsg", "sc_matmul_cbsg", "sc_cbsg_scc",
@@ -101,6 +101,8 @@ def load():
     lib.sc_profile_enable.argtypes = [vp, i32]
     lib.sc_profile_read.argtypes = [vp, c.POINTER(c.c_float)]
     lib.sc_launch_count.argtypes = [vp, c.POINTER(i64)]
+    lib.sc_last_core_selected.argtypes = [vp, c.POINTER(i32)]
+    lib.sc_last_core_selected.restype = c.c_int
     lib.sc_assign_lengths_static.argtypes = [vp, i64, i32, f64, i32, i32, vp, vp, vp, vp]
     lib.sc_assign_lengths_static.restype = c.c_int
     for name in ("sc_create", "sc_destroy", "sc_device_status", "sc_row_stats", "sc_assign_lengths",
@@ -299,6 +301,12 @@ def sc_profile_read(ctx) -> dict:
     ms = (ctypes.c_float * 8)()
     _check(load().sc_profile_read(ctx, ms), "sc_profile_read")
     return {name: float(ms[k]) for k, name in enumerate(PROFILE_PHASES) if name != "reserved"}
+
+
+def sc_last_core_selected(ctx) -> int:
+    v = ctypes.c_int32(0)
+    _check(load().sc_last_core_selected(ctx, ctypes.byref(v)), "sc_last_core_selected")
+    return int(v.value)
 
 
 def sc_launch_count(ctx) -> int:

@@ -761,6 +761,15 @@ sc_status sc_launch_count(sc_ctx *ctx, int64_t *count_host)
     return SC_OK;
 }
 
+sc_status sc_last_core_selected(sc_ctx *ctx, int32_t *pair_host)
+{
+    if (!ctx || !pair_host) return SC_ERR_ARG;
+    sc_ctx_impl *c = reinterpret_cast<sc_ctx_impl *>(ctx);
+    if (cudaDeviceSynchronize() != cudaSuccess) return SC_ERR_CUDA;
+    if (cudaMemcpy(pair_host, c->scratch + kSlotPairSelected, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) return SC_ERR_CUDA;
+    return SC_OK;
+}
+
 int32_t sc_selftest_comparator(void)
 {
     int32_t mismatches = 0;

@@ -13,10 +13,13 @@
 // one-SM core (both kernels are launched, the one not selected returns at once: the choice is device data).
 //
 // Synchronisation across the pair: "stage full" and "accumulator free" barriers live in the leader and receive remote
-// arrivals (release / acquire at cluster scope) from the other CTA's warps; "stage free" and "accumulator full" are signalled in
-// BOTH CTAs by one multicast tcgen05.commit of the issuing thread.  Each CTA loads its own half of the weight tile with its
-// own TMA loads (no multicast loads anywhere).  Every wait is bounded; a wait that runs out sets SC_ERR_TIMEOUT, raises the
-// abort flag of both CTAs, all roles drain, both CTAs meet at the cluster barrier and free their tensor memory.
+// arrivals from the other CTA's warps (plain arrivals: see p_arrive_cta; the waits acquire at cluster scope); "stage free" and
+// "accumulator full" are signalled in BOTH CTAs by one multicast tcgen05.commit of the issuing thread.  Each CTA loads its
+// own half of the weight tile with its own TMA loads (no multicast loads anywhere).  Every wait is bounded; a wait that runs
+// out sets SC_ERR_TIMEOUT, raises the abort flag of both CTAs, all roles drain, both CTAs meet at the cluster barrier and
+// free their tensor memory.
+// Epilogue: a piece that is a whole tile overwrites the zeroed outputs with plain stores; a piece of a cut tile adds its
+// share with bulk reductions (several times dearer for the warp: with one accumulator the MMAs wait for it).
 #include <type_traits>
 
 #include "sc_device.cuh"
@@ -99,8 +102,8 @@ __device__ __forceinline__ void p_cluster_sync()
 // tcgen05.wait and tcgen05.fence::before_thread_sync.  Operand W is written by ordinary stores to the ARRIVING CTA's own
 // shared memory and published to the async proxy by fence.proxy.async before the arrival; the two-SM MMA reads each CTA's
 // half of W from that CTA's own shared memory, so the leader's issuing thread passes on only the barrier's phase.  A release
-// at cluster scope would add a fence that costs each expander warp a round trip beyond the SM per stage: measured, 13 - 20 %
-// of the kernel's time, all of it on the W side, which is the critical path.
+// at cluster scope adds a fence that costs each expander warp a quarter of its time: measured, 13 - 20 % of the kernel's
+// time, all of it on the W side, which is the critical path.
 __device__ __forceinline__ void p_arrive_cta(uint32_t bar, uint32_t cta)
 {
     asm volatile("{\n\t.reg .b32 ra;\n\tmapa.shared::cluster.u32 ra, %0, %1;\n\t"
@@ -541,10 +544,9 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
                 it.op = (uint32_t)(group - kPAGroups); it.j = group - kPAGroups; it.src += (int64_t)(group - kPAGroups) * stage_stride;
                 advance(it);
             }
-            // Two register sets take turns.  The words of a stage are requested right AFTER the group's previous hand-over and
-            // used two hand-overs later: a hand-over (the release of the barrier arrival) waits for the thread's loads in
-            // flight, so loads issued just before it would hold it up for most of their latency (measured: a quarter of the
-            // expander's time), and this way they have a whole period of the group to land.
+            // Two register sets take turns.  The words of a stage are requested right after the group's previous hand-over and
+            // used two hand-overs later: they have a whole period of the group to land, and no load of the thread is in flight
+            // when it arrives on the barrier.
             uint32_t w0[kPStagePp], w1[kPStagePp], s0[kSignWords], s1[kSignWords];
             uint32_t op0 = it.op, op1 = 0u;
             bool v0 = it.valid, v1 = false;

@@ -47,6 +47,7 @@ enum ScratchSlot : int {
     kSlotRealizedTotal = 6, // int64 (slots 6,7): total assigned length
     kSlotTimeoutSite = 8,   // slots 8-10: where the first bounded wait of the tensor-core core ran out
     kSlotAnyNegA = 11,      // unipolar: set by the encode of A when any stream bit carries a negative sign
+    kSlotPairSelected = 12, // the plan of the current call selected the two-SM tensor-core kernel
     kSlotCount = 16
 };
 

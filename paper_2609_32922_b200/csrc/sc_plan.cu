@@ -138,6 +138,7 @@ __device__ void finish_plan(int32_t n_row_tiles, int32_t n_col_tiles, int32_t ta
         plan->pad[0] = use_pair;                      // which tensor-core core runs: 1 = the two-SM core
         plan->pad[1] = charge;                        // virtual units in front of every (row tile, column tile) in the prefix sums
         scratch[kSlotTicket] = 0;
+        scratch[kSlotPairSelected] = use_pair;
         scratch[kSlotAnyNegA] = 0;                    // the encode of A sets it again if it meets a negative element
         scratch[kSlotLmaxActual] = longest / planes_per_len;
     }
