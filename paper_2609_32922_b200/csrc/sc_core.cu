@@ -369,6 +369,21 @@ bool make_plane_map(CUtensorMap *map, const uint32_t *base, int64_t row_words, i
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map of the int32 accumulators [rows][cols] for bulk tensor reductions of 32 x 32 boxes staged in shared memory in
+// the 128-byte swizzle (16-byte chunk c of box row r at chunk c ^ (r & 7): conflict-free 16-byte stores by one lane per row).
+// Needs a 16-byte aligned base and cols % 4 == 0 (the row stride in bytes is a multiple of 16).
+bool make_acc_map(CUtensorMap *map, int32_t *acc, int64_t rows, int64_t cols)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn || (cols & 3) != 0 || (reinterpret_cast<uintptr_t>(acc) & 15u) != 0) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * sizeof(int32_t)};
+    cuuint32_t box[2] = {32u, 32u};
+    cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_INT32, 2, acc, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 constexpr size_t kCoreSmem = (size_t)kStages * kStageBytes + kStages * 8 + (2 * kTileM + 4) * sizeof(int32_t);
 
 template <int kMode, bool kCsa>

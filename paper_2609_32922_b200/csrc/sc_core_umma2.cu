@@ -84,6 +84,7 @@ struct PairDev {
     int32_t force;                    // run whatever the plan selected
     const uint32_t *w_sign, *a_sign;  // unipolar: nibble sign words
     int64_t n_pad;
+    int32_t acc_map_ok;               // the tensor map of the accumulators is valid (aligned, N % 4 == 0)
 };
 
 __device__ __forceinline__ uint32_t p_cluster_rank()
@@ -203,7 +204,7 @@ __device__ __forceinline__ PItem p_piece(const int32_t *s_prefix, int32_t n_pair
 
 template <int kMode>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
-core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
+core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_acc, PairDev p)
 {
     const PlanHeader plan = *p.plan;
     if (!p.force && plan.pad[0] == 0) return;              // the plan chose the one-SM core (same decision in every CTA)
@@ -388,6 +389,17 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
                 // nothing of this row in the chunk: its stream ends at or before the first position block of the chunk
                 if (__ldg(p.l_sorted + r) <= it.q0 / (p.pos_block * ppl) * p.pos_block) src = -1;
             }
+            // A cut piece whose 32 rows of this warp are consecutive rows of the output (uniform or grouped lengths: the stable
+            // sort keeps them together) adds each 32 x 32 chunk with ONE bulk tensor reduction instead of 32 row pieces.
+            int32_t run_row = -1;
+            if (p.acc_map_ok && !it.whole) {
+                const unsigned valid = __ballot_sync(0xFFFFFFFFu, src >= 0);
+                if (valid != 0u) {
+                    const int first = __ffs((int)valid) - 1;
+                    const int32_t ref = __shfl_sync(0xFFFFFFFFu, src, first) - first;
+                    if (ref >= 0 && __all_sync(0xFFFFFFFFu, src < 0 || src == ref + lane)) run_row = ref;
+                }
+            }
             if (!u_mbar_wait_warp(bar(kPAccFull), acc_cnt & 1u, s_abort, lane)) { if (lane == 0) give_up(5, acc_cnt, 0); break; }
             u_fence_after();
             if (__any_sync(0xFFFFFFFFu, src >= 0)) {
@@ -399,6 +411,7 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
                     for (int k = 0; k < 32; ++k) v[k] = (uint32_t)__float2int_rn(__uint_as_float(v[k]));   // exact fp32 integers
                     uint32_t *buf = tile0 + (chunk_cnt & 1u) * (32 * kPEpiStride);
                     asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");     // the buffer's previous reduction has read it
+                    __syncwarp();                          // ... whichever lane issued it (lane 0 issues the tensor reductions)
                     const int64_t col0 = (int64_t)it.ct * kPN + c * 32;
                     if (it.whole) {
                         // No other piece adds to this tile: the zeroed outputs are simply overwritten, straight from the
@@ -416,6 +429,20 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
                                     if (col0 + k < p.N) row[k] = (int32_t)v[k];
                             }
                         }
+                    } else if (run_row >= 0 && col0 < p.N) {
+                        // (rows of the warp without a stream in this piece hold zeros or do not exist: a lane without a row
+                        // adds nothing; rows and columns beyond the matrix are clipped by the tensor map)
+                        uint8_t *dense = reinterpret_cast<uint8_t *>(tile0) + (chunk_cnt & 1u) * 5120u;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            *reinterpret_cast<uint4 *>(dense + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                                src >= 0 ? make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]) : make_uint4(0u, 0u, 0u, 0u);
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                        if (lane == 0)
+                            asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+                                         ::"l"(reinterpret_cast<uint64_t>(&map_acc)), "r"((int32_t)col0), "r"(run_row), "r"(u_smem(dense))
+                                         : "memory");
                     } else if (bulk_ok && col0 + 32 <= p.N) {
                         uint4 *dst = reinterpret_cast<uint4 *>(buf + lane * kPEpiStride);
 #pragma unroll
@@ -674,6 +701,7 @@ core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, PairDev p)
 
 bool make_plane_map(CUtensorMap *map, const uint32_t *base, int64_t row_words, int64_t planes, int box_words,
                     int box_planes);
+bool make_acc_map(CUtensorMap *map, int32_t *acc, int64_t rows, int64_t cols);
 
 // Clusters of two CTAs of the pair kernel that can be resident at once (one CTA per SM): the grid is sized to that.
 template <int kMode>
@@ -722,10 +750,12 @@ cudaError_t launch_core_umma_pair(const CoreArgs &a, int clusters, bool force, c
     dev.n_col_tiles = (int32_t)((a.N + kPN - 1) / kPN);
     dev.force = force ? 1 : 0;
     dev.w_sign = a.w_sign; dev.a_sign = a.a_sign; dev.n_pad = a.n_pad;
+    CUtensorMap macc = mw;                                 // (a valid map in any case; used only if acc_map_ok)
+    dev.acc_map_ok = make_acc_map(&macc, a.acc, a.M, a.N) ? 1 : 0;
     if (a.mode == SC_UNIPOLAR_AND && (a.pos_block != kPosBlockSigned || !a.w_sign || !a.a_sign)) return cudaErrorInvalidValue;
     if (a.mode != SC_UNIPOLAR_AND && a.pos_block != 1) return cudaErrorInvalidValue;
-    if (a.mode == SC_UNIPOLAR_AND) core_umma_pair_kernel<SC_UNIPOLAR_AND><<<2 * clusters, kPThreads, kPairSmem, st>>>(mw, dev);
-    else core_umma_pair_kernel<SC_BIPOLAR_XNOR><<<2 * clusters, kPThreads, kPairSmem, st>>>(mw, dev);
+    if (a.mode == SC_UNIPOLAR_AND) core_umma_pair_kernel<SC_UNIPOLAR_AND><<<2 * clusters, kPThreads, kPairSmem, st>>>(mw, macc, dev);
+    else core_umma_pair_kernel<SC_BIPOLAR_XNOR><<<2 * clusters, kPThreads, kPairSmem, st>>>(mw, macc, dev);
     count_launches(1);
     return cudaGetLastError();
 }

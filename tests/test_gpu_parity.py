@@ -161,6 +161,24 @@ def test_sm_pair_core_whole_tile_pieces(sc, binding, oracle, N):
     assert sc.device_status() == 0
 
 
+@pytest.mark.parametrize("mode", ["bipolar", "unipolar"])
+def test_sm_pair_core_cut_pieces_of_consecutive_rows(sc, binding, oracle, mode):
+    """The two-SM core on uniform lengths with few tiles (every piece is a cut tile): warps whose 32 rows are consecutive rows
+    of the output add each 32 x 32 chunk with one bulk tensor reduction.  The shape puts rows beyond M and columns beyond N
+    inside boxes (clipped), N % 32 != 0 with N % 4 == 0, and a block of rows without a stream splits one warp's run (that warp
+    takes the row-by-row path) and leaves lanes without a row in the last tile.  Every entry against the oracle."""
+    M, N = 1100, 1020
+    w, L_rows = wl.small_ragged(seed=23, M=M, K=100, N=N, mode=mode, Lmin=56, Lmax=56)
+    L_rows[:] = 56
+    L_rows[300:340] = 0
+    A, W = wl.make_inputs(w)
+    P, C = T.gpu_matmul(sc, binding, w, A, W, L_rows, 56, core=5)
+    ref = T.oracle_matmul(oracle, w, A, W, L_rows)
+    assert np.array_equal(P, ref["P"])
+    assert T.close_enough(C, ref["C"])
+    assert sc.device_status() == 0
+
+
 def test_groups_and_accumulator_workspace(sc, binding, oracle):
     """Lengths per group of 8 rows (last group short); P not requested (accumulators live in the workspace)."""
     w, _ = wl.small_ragged(seed=5, M=150, K=96, N=130)
