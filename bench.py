@@ -36,8 +36,8 @@ L2_FLUSH_BYTES = 256 << 20
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one core-kernel launch, from an
 # `ncu --set full` capture of this command on the workload named by the key.
-NCU_CORE_TRAFFIC_BYTES = {("vit_b16_fc1", "alu"): 85.4e6, ("vit_b16_fc1", "umma"): 93.8e6,
-                          ("vit_l14_fc1_L128", "umma"): 5.35e9}
+NCU_CORE_TRAFFIC_BYTES = {("vit_b16_fc1", "alu"): 85.4e6, ("vit_b16_fc1", "umma"): 93.8e6, ("vit_b16_fc1", "pair"): 93.9e6,
+                          ("vit_l14_fc1_L128", "pair"): 7.21e9}
 
 FP4_TO_BF16_NOMINAL = 4.0       # dense tensor peaks: 9 PFLOP/s fp4 vs 2.25 PFLOP/s bf16
 
@@ -58,7 +58,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--config", default="vit_b16_fc1", help="workload name (see workloads.all_configs)")
-    ap.add_argument("--core", type=int, default=0, help="GEMM core variant (0 auto, 1 popc, 2 carry-save)")
+    ap.add_argument("--core", type=int, default=0, help="GEMM core variant (0 auto, 1 popc, 2 carry-save, 3 simple, 4 one-SM tensor core, "
+                    "5 two-SM tensor core)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch the step's kernels one by one instead of replaying "
@@ -661,7 +662,7 @@ def main():
     core_avg_ms = statistics.mean(core_ms)
     achieved = bitops_per_step / (core_avg_ms * 1e-3)                    # stream bit-ops (= 1-bit MACs) per second
     alu_peak = POPC_PER_CLK_PER_SM * 32.0 * n_sm * sm_max * 1e6          # POPC-pipe bound of the ALU cores
-    uses_tensor = args.core in (0, 4) and w.K * Lmax <= (1 << 24)
+    uses_tensor = args.core in (0, 4, 5) and w.K * Lmax <= (1 << 24)
     if uses_tensor:
         # Tensor contraction: one stream bit-op is one multiply-accumulate = 2 ops, run as 4-bit floating point
         # (e2m1, tcgen05.mma kind::mxf4).  Two denominators: (a) the measured bf16 burst figure x the nominal ratio of the
