@@ -43,7 +43,7 @@ constexpr int kPEpiFirstWarp = 2, kPEpiWarps = 4;
 constexpr int kPAGroups = 3, kPAFirstWarp = 6, kPAWarps = 4;
 constexpr int kPWGroups = 3, kPWCols = 2, kPWWarps = kPH / (32 * kPWCols);
 constexpr int kPWFirstWarp = kPAFirstWarp + kPAGroups * kPAWarps;
-constexpr int kPIssuers = 3;
+constexpr int kPIssuers = 2;
 constexpr int kPIssuerBWarp = kPWFirstWarp + kPWGroups * kPWWarps;
 constexpr int kPThreads = 32 * (kPIssuerBWarp + kPIssuers - 1);
 static_assert(kPOpStages % kPIssuers == 0 && kPOpStages % kPAGroups == 0 && kPOpStages % kPWGroups == 0,
