@@ -40,15 +40,15 @@ constexpr int kPOpStages = 6;                  // depth of both operand rings
 constexpr int kPStagePp = kPOpSteps * 2;       // planes of one operand stage
 constexpr int kPOpsPerRaw = kStagePlanes / kPStagePp;
 constexpr int kPEpiFirstWarp = 2, kPEpiWarps = 4;
-constexpr int kPAGroups = 3, kPAFirstWarp = 6, kPAWarps = 4;
+constexpr int kPAFirstWarp = 6, kPAWarps = 4;    // activation expanders: kAG groups (a template parameter: 3, or 2 for short calls) of 4 warps
 constexpr int kPWGroups = 3, kPWCols = 2, kPWWarps = kPH / (32 * kPWCols);
-constexpr int kPWFirstWarp = kPAFirstWarp + kPAGroups * kPAWarps;
+__host__ __device__ constexpr int p_w_first_warp(int ag) { return kPAFirstWarp + ag * kPAWarps; }
 constexpr int kPIssuers = 2;
-constexpr int kPIssuerBWarp = kPWFirstWarp + kPWGroups * kPWWarps;
-constexpr int kPThreads = 32 * (kPIssuerBWarp + kPIssuers - 1);
-static_assert(kPOpStages % kPIssuers == 0 && kPOpStages % kPAGroups == 0 && kPOpStages % kPWGroups == 0,
+__host__ __device__ constexpr int p_issuer_b_warp(int ag) { return p_w_first_warp(ag) + kPWGroups * kPWWarps; }
+__host__ __device__ constexpr int p_threads(int ag) { return 32 * (p_issuer_b_warp(ag) + kPIssuers - 1); }
+static_assert(kPOpStages % kPIssuers == 0 && kPOpStages % 3 == 0 && kPOpStages % 2 == 0 && kPOpStages % kPWGroups == 0,
               "issuers and expander groups own fixed ring slots");
-static_assert(kPAFirstWarp % 4 == 2 && kPAWarps == 4 && kPStagePp == kPosBlockSigned && kPThreads <= 1024, "role layout");
+static_assert(kPAFirstWarp % 4 == 2 && kPAWarps == 4 && kPStagePp == kPosBlockSigned && p_threads(3) <= 1024, "role layout");
 
 constexpr uint32_t kPRawStageBytes = kPRawPlanes * kPH * 4;     // 24 KB
 constexpr uint32_t kPLbo = kPH * 16;                            // bytes between the two 16-byte K chunks of a K-step
@@ -59,6 +59,7 @@ constexpr uint32_t kPTmemCols = 512;
 constexpr uint32_t kPARingCol = kPN;                            // accumulator: columns 0 .. 255
 constexpr uint32_t kPSfCol = 448, kPSfCols = 64;                // scale factors (every byte 2^0): A's at 448, B's at 480
 static_assert(kPARingCol + kPOpStages * kPOpSteps * 8 <= kPSfCol && kPSfCol + kPSfCols == kPTmemCols, "tensor memory budget");
+constexpr int kPShortCallStages = 1024;                         // below this many stages per CTA pair: two activation expander groups
 constexpr int kPMaxPairs = 1024;                                // row-tile pairs whose unit prefix fits the shared-memory table
 
 // "stage full" is four barriers per ring slot -- the activation and the weight expanders of either CTA arrive on a
@@ -202,10 +203,14 @@ __device__ __forceinline__ PItem p_piece(const int32_t *s_prefix, int32_t n_pair
     return it;
 }
 
-template <int kMode>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
+// kAG: groups of activation expander warps.  Three keep up with long pieces; with two the CTA is 22 warps instead of 26, which
+// is 1 - 3 % faster on calls of a few hundred stages per CTA pair (measured: config 2 0.204 -> 0.198 ms) and 1.5 - 3 % slower on
+// long ones; the host picks by the stages a pair can get at most.
+template <int kMode, int kAG>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(p_threads(kAG), 1)
 core_umma_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_acc, PairDev p)
 {
+    constexpr int kPAGroups = kAG, kPWFirstWarp = p_w_first_warp(kAG), kPIssuerBWarp = p_issuer_b_warp(kAG), kPThreads = p_threads(kAG);
     const PlanHeader plan = *p.plan;
     if (!p.force && plan.pad[0] == 0) return;              // the plan chose the one-SM core (same decision in every CTA)
     const int32_t n_pairs = (plan.n_row_tiles + 1) / 2;
@@ -704,16 +709,16 @@ bool make_plane_map(CUtensorMap *map, const uint32_t *base, int64_t row_words, i
 bool make_acc_map(CUtensorMap *map, int32_t *acc, int64_t rows, int64_t cols);
 
 // Clusters of two CTAs of the pair kernel that can be resident at once (one CTA per SM): the grid is sized to that.
-template <int kMode>
-static cudaError_t pair_clusters_mode(int sm_count, int *clusters)
+template <int kMode, int kAG>
+static cudaError_t pair_clusters_variant(int sm_count, int *clusters)
 {
     static int cached = -1;
     if (cached < 0) {
-        cudaError_t e = cudaFuncSetAttribute(core_umma_pair_kernel<kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmem);
+        cudaError_t e = cudaFuncSetAttribute(core_umma_pair_kernel<kMode, kAG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmem);
         if (e != cudaSuccess) return e;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(sm_count / 2 * 2));
-        cfg.blockDim = dim3(kPThreads);
+        cfg.blockDim = dim3(p_threads(kAG));
         cfg.dynamicSmemBytes = kPairSmem;
         cudaLaunchAttribute attr;
         attr.id = cudaLaunchAttributeClusterDimension;
@@ -721,11 +726,24 @@ static cudaError_t pair_clusters_mode(int sm_count, int *clusters)
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
         int n = 0;
-        e = cudaOccupancyMaxActiveClusters(&n, core_umma_pair_kernel<kMode>, &cfg);
+        e = cudaOccupancyMaxActiveClusters(&n, core_umma_pair_kernel<kMode, kAG>, &cfg);
         if (e != cudaSuccess) return e;
         cached = n < sm_count / 2 ? n : sm_count / 2;
     }
     *clusters = cached;
+    return cudaSuccess;
+}
+
+// (the smaller of the two variants' counts: the plan is built before the variant is picked)
+template <int kMode>
+static cudaError_t pair_clusters_mode(int sm_count, int *clusters)
+{
+    int c3 = 0, c2 = 0;
+    cudaError_t e = pair_clusters_variant<kMode, 3>(sm_count, &c3);
+    if (e != cudaSuccess) return e;
+    e = pair_clusters_variant<kMode, 2>(sm_count, &c2);
+    if (e != cudaSuccess) return e;
+    *clusters = c3 < c2 ? c3 : c2;
     return cudaSuccess;
 }
 
@@ -754,8 +772,17 @@ cudaError_t launch_core_umma_pair(const CoreArgs &a, int clusters, bool force, c
     dev.acc_map_ok = make_acc_map(&macc, a.acc, a.M, a.N) ? 1 : 0;
     if (a.mode == SC_UNIPOLAR_AND && (a.pos_block != kPosBlockSigned || !a.w_sign || !a.a_sign)) return cudaErrorInvalidValue;
     if (a.mode != SC_UNIPOLAR_AND && a.pos_block != 1) return cudaErrorInvalidValue;
-    if (a.mode == SC_UNIPOLAR_AND) core_umma_pair_kernel<SC_UNIPOLAR_AND><<<2 * clusters, kPThreads, kPairSmem, st>>>(mw, macc, dev);
-    else core_umma_pair_kernel<SC_BIPOLAR_XNOR><<<2 * clusters, kPThreads, kPairSmem, st>>>(mw, macc, dev);
+    // Stages a CTA pair gets at most (every row at Lmax): short calls run the variant with two activation expander groups.
+    const int64_t pairs = (a.m_pad / kTileM + 1) / 2;
+    const int64_t units = ((int64_t)a.Lmax * a.kw + kStagePlanes - 1) / kStagePlanes;
+    const bool short_call = pairs * dev.n_col_tiles * units * kPOpsPerRaw / clusters < kPShortCallStages;
+    if (a.mode == SC_UNIPOLAR_AND) {
+        if (short_call) core_umma_pair_kernel<SC_UNIPOLAR_AND, 2><<<2 * clusters, p_threads(2), kPairSmem, st>>>(mw, macc, dev);
+        else core_umma_pair_kernel<SC_UNIPOLAR_AND, 3><<<2 * clusters, p_threads(3), kPairSmem, st>>>(mw, macc, dev);
+    } else {
+        if (short_call) core_umma_pair_kernel<SC_BIPOLAR_XNOR, 2><<<2 * clusters, p_threads(2), kPairSmem, st>>>(mw, macc, dev);
+        else core_umma_pair_kernel<SC_BIPOLAR_XNOR, 3><<<2 * clusters, p_threads(3), kPairSmem, st>>>(mw, macc, dev);
+    }
     count_launches(1);
     return cudaGetLastError();
 }
