@@ -172,11 +172,12 @@ encode_kernel(const __grid_constant__ PhiloxKeys ks, const __grid_constant__ Enc
         uint32_t out_pos[8];
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
-            out_pos[t] = 0u;
-            if (blk * 32 >= (info[t] >> 10)) continue;                 // warp-uniform: the row has ended
+            // (no branch per row: the eight rows' Philox chains and shuffle butterflies are independent and interleave;
+            // a row that has ended -- rows of a group are neighbours in the order of lengths -- is computed and dropped)
             const uint32_t z = sng_word(ks, p.stream_word, elem[t], (uint32_t)blk, info[t] & 0x1FF);
             // 32 x 32 bit transpose across the warp: lane b receives position b of the 32 depth elements
-            out_pos[t] = transpose(z);
+            const uint32_t zt = transpose(z);
+            out_pos[t] = blk * 32 < (info[t] >> 10) ? zt : 0u;
         }
         const int32_t l = blk * 32 + lane;                             // the position this lane holds
         if (l < l_write) {
