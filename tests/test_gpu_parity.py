@@ -473,6 +473,25 @@ def test_all_rows_without_a_stream(sc, binding, oracle, core):
     assert (P == 0).all() and (C == 0).all()
 
 
+def test_selected_tensor_core_kernel_is_reported(sc, binding):
+    """`sc_last_core_selected`: forced choices are reported as forced, the integer cores report 0, and under AUTO the plan picks the
+    two-SM kernel for long uniform streams and the one-SM kernel for a few positions per row (both decided on the device from
+    the lengths), with identical counts either way."""
+    w, L_rows = wl.small_ragged(seed=61, M=1024, K=1024, N=1024, mode="bipolar", Lmin=96, Lmax=96)
+    A, W = wl.make_inputs(w)
+    L_long = np.full(1024, 96, dtype=np.int32)
+    L_short = np.full(1024, 2, dtype=np.int32)
+    seen = {}
+    for core, L in ((4, L_long), (5, L_long), (2, L_long), (0, L_long), (0, L_short)):
+        P, _ = T.gpu_matmul(sc, binding, w, A, W, L, 96, core=core)
+        seen[(core, int(L[0]))] = (binding.sc_last_core_selected(sc.ctx), P)
+    assert seen[(4, 96)][0] == 0 and seen[(5, 96)][0] == 1 and seen[(2, 96)][0] == 0
+    assert seen[(0, 96)][0] == 1 and seen[(0, 2)][0] == 0
+    for key in ((5, 96), (2, 96), (0, 96)):
+        assert np.array_equal(seen[(4, 96)][1], seen[key][1]), key
+    assert sc.device_status() == 0
+
+
 @pytest.mark.parametrize("name", ["vit_b16_fc1", "vit_b16_qkv_mixed", "dit_xl2_linear_grouped", "vit_l14_fc2_L32"])
 def test_cores_agree_on_every_output_and_repeat(sc, binding, oracle, name):
     """Full-size runs: the tensor-core core and the carry-save integer core share no code after the encode, so
