@@ -92,6 +92,7 @@ class ClockSampler:
         self.gpu_index = gpu_index
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
+        self._first = threading.Event()          # set once the first sample has landed (or sampling is impossible)
         self._thread = None
 
     def _physical_index(self):
@@ -110,6 +111,7 @@ class ClockSampler:
         self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
         while not self._stop.is_set():
             self.samples.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+            self._first.set()
             try:
                 bits = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
             except Exception:
@@ -131,10 +133,12 @@ class ClockSampler:
                 f = [x.strip() for x in out.strip().split(",")]
                 self.samples.append(float(f[0]))
                 self.max_mhz = float(f[1])
+                self._first.set()
                 for name, val in zip(names, f[2:6]):
                     if val.lower().startswith("active"):
                         self.reasons.add(name)
             except Exception:
+                self._first.set()
                 return
 
     def _run(self):
@@ -142,11 +146,14 @@ class ClockSampler:
             self._run_nvml()
         except Exception:
             self._run_smi()
+        self._first.set()
 
     def start(self):
         self._thread = threading.Thread(target=self._run, daemon=True)
         self._thread.start()
-        time.sleep(0.02)          # let the first sample land before the timed region starts
+        # The first sample must land before the timed region starts: loading NVML in a cold process can take longer than a
+        # short timed region lasts, which would leave the run without a clock record.
+        self._first.wait(timeout=20.0)
 
     def stop(self):
         self._stop.set()

@@ -196,7 +196,9 @@ sc_status sc_create(sc_ctx **ctx_out, int device)
     if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->ev_plan, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_a_done, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_rows_done, cudaEventDisableTiming) != cudaSuccess) {
         cudaFree(c->scratch); delete c; return SC_ERR_CUDA;
     }
     c->overlap = true;
@@ -213,6 +215,7 @@ sc_status sc_destroy(sc_ctx *ctx)
     cudaEventDestroy(c->ev1);
     for (int k = 0; k < SC_PROFILE_PHASES; ++k) cudaEventDestroy(c->phase_ev[k]);
     cudaEventDestroy(c->ev_fork); cudaEventDestroy(c->ev_plan); cudaEventDestroy(c->ev_join);
+    cudaEventDestroy(c->ev_a_done); cudaEventDestroy(c->ev_rows_done);
     cudaStreamDestroy(c->side);
     cudaFree(c->scratch);
     delete c;
@@ -480,7 +483,16 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     ca.acc = acc; ca.scratch = c->scratch; ca.sm_count = c->sm_count; ca.Lmax = Lmax;
     ca.pop_a = reinterpret_cast<int32_t *>(base + w.pop_a);
     ca.pop_w = pop_w;
-    if (and_form && launch_row_corrections(ca, st) != cudaSuccess) return SC_ERR_CUDA;   // counted with the W encode phase
+    // The row popcounts of A feed the decode only: they run on the side stream beside the core (their small CTAs fit on
+    // the SMs next to the core's one CTA each), forked after the encode of A and joined before the decode.
+    const bool fork_rows = and_form && c->overlap && !c->profiling;
+    if (fork_rows) {
+        if (cudaEventRecord(c->ev_a_done, st) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_a_done, 0) != cudaSuccess ||
+            launch_row_corrections(ca, c->side) != cudaSuccess || cudaEventRecord(c->ev_rows_done, c->side) != cudaSuccess)
+            return SC_ERR_CUDA;
+    } else if (and_form && launch_row_corrections(ca, st) != cudaSuccess) {
+        return SC_ERR_CUDA;                                                              // counted with the W encode phase
+    }
     mark(4);
     if (umma) {
         // both kernels are enqueued; the one the plan did not select returns at once
@@ -491,6 +503,7 @@ static sc_status matmul_impl(sc_ctx *ctx, const float *A, const float *W, const 
     }
 
     mark(5);
+    if (fork_rows && cudaStreamWaitEvent(st, c->ev_rows_done, 0) != cudaSuccess) return SC_ERR_CUDA;
     // a8: decode
     if (and_form) {
         if (launch_decode_and(acc, Mt, N, K, w.n_pad, l_rows, ca.pop_a, ca.pop_w, sigma_a, sigma_w, P, C, st, M,

@@ -61,7 +61,7 @@ struct sc_ctx_impl {
     cudaEvent_t phase_ev[SC_PROFILE_PHASES];
     // the W-side work of a call (scales, encode, popcount tables) runs on a side stream beside the A-side work
     cudaStream_t side;
-    cudaEvent_t ev_fork, ev_plan, ev_join;
+    cudaEvent_t ev_fork, ev_plan, ev_join, ev_a_done, ev_rows_done;
     bool overlap;
 };
 
