@@ -168,8 +168,29 @@ encode_kernel(const __grid_constant__ PhiloxKeys ks, const __grid_constant__ Enc
     }
 
     // ---- phase 2: the blocks ----
+    // (as far as the longest of the warp's eight rows reaches: groups of rows that do not exist -- the padding of a batched
+    // product -- or that have all ended write zeros below without drawing anything)
+    int32_t live_len = 0;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) live_len = max(live_len, info[t] >> 10);
+    const int32_t blk_live = min(blk1, (live_len + 31) >> 5);
 #pragma unroll 1
     for (int32_t blk = blk0; blk < blk1; ++blk) {
+        if (blk >= blk_live) {                                         // warp-uniform
+            const int32_t l = blk * 32 + lane;
+            if (l < l_write) {
+                const int64_t plane = plane_index_pow2(l, w, p.kw, p.pos_shift) * p.ppq;
+                uint4 *dst = reinterpret_cast<uint4 *>(p.streams + plane * p.r_pad + r0);
+                dst[0] = make_uint4(0u, 0u, 0u, 0u);
+                dst[1] = make_uint4(0u, 0u, 0u, 0u);
+                if (kMode == SC_UNIPOLAR_AND && p.ppq == 2) {
+                    uint4 *dn = reinterpret_cast<uint4 *>(p.streams + (plane + 1) * p.r_pad + r0);
+                    dn[0] = make_uint4(0u, 0u, 0u, 0u);
+                    dn[1] = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+            continue;
+        }
         uint32_t out_pos[8];
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
