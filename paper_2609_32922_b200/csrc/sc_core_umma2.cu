@@ -59,7 +59,7 @@ constexpr uint32_t kPTmemCols = 512;
 constexpr uint32_t kPARingCol = kPN;                            // accumulator: columns 0 .. 255
 constexpr uint32_t kPSfCol = 448, kPSfCols = 64;                // scale factors (every byte 2^0): A's at 448, B's at 480
 static_assert(kPARingCol + kPOpStages * kPOpSteps * 8 <= kPSfCol && kPSfCol + kPSfCols == kPTmemCols, "tensor memory budget");
-constexpr int kPShortCallStages = 1024;                         // below this many stages per CTA pair: two activation expander groups
+constexpr int kPShortCallStages = 1024;                         // below this many stages per CTA pair (twice as many for bipolar calls): two activation expander groups
 constexpr int kPMaxPairs = 1024;                                // row-tile pairs whose unit prefix fits the shared-memory table
 
 // "stage full" is four barriers per ring slot -- the activation and the weight expanders of either CTA arrive on a
@@ -775,7 +775,8 @@ cudaError_t launch_core_umma_pair(const CoreArgs &a, int clusters, bool force, c
     // Stages a CTA pair gets at most (every row at Lmax): short calls run the variant with two activation expander groups.
     const int64_t pairs = (a.m_pad / kTileM + 1) / 2;
     const int64_t units = ((int64_t)a.Lmax * a.kw + kStagePlanes - 1) / kStagePlanes;
-    const bool short_call = pairs * dev.n_col_tiles * units * kPOpsPerRaw / clusters < kPShortCallStages;
+    const bool short_call = pairs * dev.n_col_tiles * units * kPOpsPerRaw / clusters <
+                            (a.mode == SC_UNIPOLAR_AND ? kPShortCallStages : 2 * kPShortCallStages);
     if (a.mode == SC_UNIPOLAR_AND) {
         if (short_call) core_umma_pair_kernel<SC_UNIPOLAR_AND, 2><<<2 * clusters, p_threads(2), kPairSmem, st>>>(mw, macc, dev);
         else core_umma_pair_kernel<SC_UNIPOLAR_AND, 3><<<2 * clusters, p_threads(3), kPairSmem, st>>>(mw, macc, dev);
